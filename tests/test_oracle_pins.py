@@ -1,0 +1,252 @@
+"""Pins for the CPU oracle: it is checked against what the paper and the
+mathematics fix, never against itself and never against the CUDA path.
+
+  * Corollary 1 / Appendix A.6: diagonal quadratic + plain GD + alpha = 1 makes
+    the extrapolated point the K-th GD iterate and the new point the (K+1)-th.
+  * brute force: K explicit GD steps written as Python loops.
+  * identities of the scale factor (Eq. (scale_factor), Eq. (geom_sum_def)).
+  * AdamW: a library AdamW in float64, and the closed form of its first step.
+  * norm: closed forms and a library norm.
+"""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import gxpo_oracle as ora
+from paper_2605_06755_b200 import workloads
+
+
+def quad_grad_fn(a, b):
+    a64, b64 = a.astype(np.float64), b.astype(np.float64)
+    return lambda which, theta: a64 * theta - b64
+
+
+# ---------------------------------------------------------------------------
+# Corollary 1: closed form on the diagonal-quadratic surrogate (BASELINE config 0)
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("K", [2, 3, 5, 10])
+@pytest.mark.parametrize("alpha", [1.0, 0.5, 0.1, 0.0])
+def test_closed_form_diagonal_quadratic(K, alpha):
+    n, eta = 4096, 0.1
+    a, b, theta0 = workloads.quadratic_surrogate(n, seed=0)
+    a64, b64, t64 = (x.astype(np.float64) for x in (a, b, theta0))
+    star = b64 / a64
+    r = 1.0 - eta * a64
+    st = ora.State(theta0, ora.OptCfg(kind="gd", lr=eta))
+    cfg = ora.GxpoCfg(K=K, alpha=alpha, delta=1e-8)
+    trace = {}
+    nrm = ora.active_step(st, cfg, quad_grad_fn(a, b), round_f32=False, trace=trace)
+    assert np.all(np.abs(a64 * t64 - b64) > 1e-8)          # every coordinate active
+    # the two probes are GD iterates 1 and 2
+    np.testing.assert_allclose(trace["theta1"], star + r * (t64 - star), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(trace["theta2"], star + r**2 * (t64 - star), rtol=0, atol=1e-12)
+    # extrapolated point = K-th GD iterate (Appendix A.6)
+    np.testing.assert_allclose(trace["theta_K"], star + r**K * (t64 - star), rtol=0, atol=1e-10)
+    # repositioned point for general alpha (Eq. (blend_step) applied to the above)
+    blend = 1.0 - alpha + alpha * r**K
+    np.testing.assert_allclose(trace["theta_tilde"], star + blend * (t64 - star), rtol=0, atol=1e-10)
+    # slow correction: one more GD step from theta-tilde
+    np.testing.assert_allclose(st.theta, star + r * blend * (t64 - star), rtol=0, atol=1e-10)
+    if alpha == 1.0:
+        np.testing.assert_allclose(st.theta, star + r**(K + 1) * (t64 - star), rtol=0, atol=1e-10)
+    # ||g_slow|| where g_slow = a (theta_tilde - theta*)
+    want = math.sqrt(float(np.sum((a64 * blend * (t64 - star))**2)))
+    assert nrm == pytest.approx(want, rel=1e-12)
+
+
+def test_m_active_steps_equal_m_times_K_plus_1_gd_steps():
+    n, eta, K, m_steps = 512, 0.1, 5, 20
+    a, b, theta0 = workloads.quadratic_surrogate(n, seed=3)
+    a64, b64, t64 = (x.astype(np.float64) for x in (a, b, theta0))
+    star, r = b64 / a64, 1.0 - eta * a64
+    st = ora.State(theta0, ora.OptCfg(kind="gd", lr=eta))
+    cfg = ora.GxpoCfg(K=K, alpha=1.0, delta=0.0)
+    for s in range(1, m_steps + 1):
+        ora.active_step(st, cfg, quad_grad_fn(a, b))
+        np.testing.assert_allclose(st.theta, star + r**((K + 1) * s) * (t64 - star), rtol=0,
+                                   atol=1e-9)
+
+
+@pytest.mark.parametrize("K", [2, 3, 5, 10])
+def test_brute_force_K_explicit_gd_steps(K):
+    n, eta = 16, 0.1
+    a, b, theta0 = workloads.quadratic_surrogate(n, seed=11)
+    st = ora.State(theta0, ora.OptCfg(kind="gd", lr=eta))
+    trace = {}
+    ora.active_step(st, ora.GxpoCfg(K=K, alpha=1.0, delta=1e-8), quad_grad_fn(a, b), trace=trace)
+    for i in range(n):                      # plain Python loops, coordinate by coordinate
+        x = float(theta0[i])
+        for _ in range(K):
+            x = x - eta * (float(a[i]) * x - float(b[i]))
+        assert trace["theta_K"][i] == pytest.approx(x, abs=1e-12)
+        x = x - eta * (float(a[i]) * x - float(b[i]))
+        assert st.theta[i] == pytest.approx(x, abs=1e-12)
+
+
+# ---------------------------------------------------------------------------
+# scale factor identities
+# ---------------------------------------------------------------------------
+def _scale(r, K, delta=1e-8, den_eps=0.0):
+    r = np.atleast_1d(np.asarray(r, dtype=np.float64))
+    g0 = np.ones_like(r)
+    g1 = r.copy()
+    z = np.zeros_like(r)
+    one = np.ones_like(r)
+    # theta0 = 0, theta2 = 1, alpha = 1  ->  theta_tilde = scale
+    _, _, sc = ora.extrapolate(z, one, g0, g1, K, 1.0, delta, den_eps, want_aux=True)
+    return sc
+
+
+def test_scale_identities():
+    r = np.array([-3.0, -0.5, 0.0, 0.3, 0.9, 1.0, 1.7, 4.0])
+    for K in (2, 3, 4, 5, 10):
+        np.testing.assert_allclose(_scale(1.0, K), K / 2.0, rtol=1e-15)     # S_K(1) = K
+        np.testing.assert_allclose(_scale(0.0, K), 1.0, rtol=1e-15)
+    np.testing.assert_allclose(_scale(r, 2), np.ones_like(r), rtol=1e-15)    # K = 2: observed
+    np.testing.assert_allclose(_scale(r, 3), 1.0 + r**2 / (1.0 + r), rtol=1e-14)
+    np.testing.assert_allclose(_scale(r, 4), 1.0 + r**2, rtol=1e-14)
+    rr = r[r != 1.0]
+    for K in (3, 5, 10):                    # the simplified form printed under Eq. (scale_factor)
+        np.testing.assert_allclose(_scale(rr, K), (1.0 - rr**K) / (1.0 - rr**2), rtol=1e-12)
+
+
+def test_literal_pole_at_minus_one_and_guard():
+    assert np.isposinf(_scale(-1.0, 3)[0])          # S_3(-1) / 0 = 1 / 0
+    assert np.isnan(_scale(-1.0, 4)[0])             # 0 / 0
+    assert _scale(-1.0, 3, den_eps=1e-6)[0] == 1.0  # guarded: treated as inactive
+    assert _scale(-1.0 + 1e-7, 3, den_eps=1e-6)[0] == 1.0
+    assert _scale(-1.0 + 1e-3, 3, den_eps=1e-6)[0] != 1.0
+
+
+def test_active_set_is_strict_and_inactive_keeps_two_probe_displacement():
+    delta = 1e-3
+    g0 = np.array([1e-3, -1e-3, 1.0000001e-3, 0.0, 5e-4, -2.0])
+    g1 = np.array([7.0, 7.0, 2e-3, 3.0, 1.0, -1.0])
+    theta0 = np.linspace(-1, 1, 6)
+    theta2 = theta0 + np.array([0.1, -0.2, 0.3, 0.4, -0.5, 0.6])
+    K, alpha = 5, 0.5
+    tilde, tk, sc = ora.extrapolate(theta0, theta2, g0, g1, K, alpha, delta, want_aux=True)
+    assert list(sc[[0, 1, 3, 4]]) == [1.0] * 4        # |g0| == delta is NOT active
+    assert sc[2] != 1.0 and sc[5] != 1.0
+    np.testing.assert_allclose(tk[[0, 1, 3, 4]], theta2[[0, 1, 3, 4]], rtol=1e-14)
+    np.testing.assert_allclose(tilde, theta0 + alpha * (tk - theta0), rtol=1e-15)
+    # inactive coordinates under GD keep -eta (g0 + g1): run the whole step
+    eta = 0.25
+    st = ora.State(theta0, ora.OptCfg(kind="gd", lr=eta))
+    grads = [g0, g1, np.zeros(6)]
+    trace = {}
+    ora.active_step(st, ora.GxpoCfg(K=K, alpha=1.0, delta=delta), lambda w, th: grads[w],
+                    trace=trace)
+    np.testing.assert_allclose(trace["theta_K"][[0, 1, 3, 4]],
+                               (theta0 - eta * (g0 + g1))[[0, 1, 3, 4]], rtol=1e-15)
+
+
+def test_alpha_endpoints():
+    rng = np.random.default_rng(5)
+    theta0, theta2 = rng.standard_normal(64), rng.standard_normal(64)
+    g0, g1 = rng.standard_normal(64), rng.standard_normal(64)
+    t0, tk, _ = ora.extrapolate(theta0, theta2, g0, g1, 5, 0.0, 1e-8, want_aux=True)
+    np.testing.assert_array_equal(t0, theta0)                     # alpha = 0 ignores it
+    t1, tk, _ = ora.extrapolate(theta0, theta2, g0, g1, 5, 1.0, 1e-8, want_aux=True)
+    np.testing.assert_allclose(t1, tk, rtol=1e-14)                # alpha = 1 adopts it
+
+
+def test_round_f32_rounds_once_at_the_boundary():
+    rng = np.random.default_rng(6)
+    theta0, theta2 = rng.standard_normal(256), rng.standard_normal(256)
+    g0, g1 = rng.standard_normal(256), rng.standard_normal(256)
+    exact = ora.extrapolate(theta0, theta2, g0, g1, 5, 0.5, 1e-8)
+    rounded = ora.extrapolate(theta0, theta2, g0, g1, 5, 0.5, 1e-8, round_f32=True)
+    np.testing.assert_array_equal(rounded, exact.astype(np.float32).astype(np.float64))
+
+
+# ---------------------------------------------------------------------------
+# AdamW against a library routine and a closed form
+# ---------------------------------------------------------------------------
+def test_adamw_matches_library_float64():
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(7)
+    n = 1000
+    theta = rng.standard_normal(n)
+    opt = ora.OptCfg(kind="adamw", lr=3e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    p = torch.nn.Parameter(torch.tensor(theta, dtype=torch.float64))
+    lib_opt = torch.optim.AdamW([p], lr=opt.lr, betas=(opt.beta1, opt.beta2), eps=opt.eps,
+                                weight_decay=opt.weight_decay)
+    st = ora.State(theta, opt)
+    for step in range(5):
+        g = rng.standard_normal(n) * 10.0 ** rng.integers(-6, 1, size=n)
+        p.grad = torch.tensor(g, dtype=torch.float64)
+        lib_opt.step()
+        st.optim_step(ora.as_f64(g), round_f32=False)
+        assert st.t_opt == step + 1
+        s = lib_opt.state[p]
+        np.testing.assert_allclose(st.theta, p.detach().numpy(), rtol=1e-12, atol=1e-15)
+        np.testing.assert_allclose(st.m, s["exp_avg"].numpy(), rtol=1e-12, atol=1e-300)
+        np.testing.assert_allclose(st.v, s["exp_avg_sq"].numpy(), rtol=1e-12, atol=1e-300)
+
+
+def test_adamw_first_step_is_sign_step():
+    # from m = v = 0 with no decay: m_hat = g, v_hat = g^2, update = lr g / (|g| + eps)
+    g = np.array([3.0, -0.5, 1e-3, -20.0])
+    theta = np.array([1.0, 2.0, -3.0, 0.25])
+    opt = ora.OptCfg(kind="adamw", lr=0.1, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0)
+    st = ora.State(theta, opt)
+    st.optim_step(g, round_f32=False)
+    np.testing.assert_allclose(st.theta, theta - 0.1 * g / (np.abs(g) + 1e-8), rtol=1e-12)
+    np.testing.assert_allclose(st.m, 0.1 * g, rtol=1e-12)
+    np.testing.assert_allclose(st.v, 0.001 * g * g, rtol=1e-12)
+
+
+def test_adamw_weight_decay_is_decoupled():
+    # zero gradient from zero state: only the decay acts, theta <- theta (1 - lr wd)
+    theta = np.array([2.0, -4.0])
+    opt = ora.OptCfg(kind="adamw", lr=0.5, weight_decay=0.1)
+    st = ora.State(theta, opt)
+    st.optim_step(np.zeros(2), round_f32=False)
+    np.testing.assert_allclose(st.theta, theta * 0.95, rtol=1e-15)
+
+
+def test_active_step_advances_optimizer_state_three_times():
+    rng = np.random.default_rng(8)
+    n = 64
+    opt = ora.OptCfg(kind="adamw", lr=1e-3)
+    st = ora.State(rng.standard_normal(n), opt)
+    gs = [rng.standard_normal(n) for _ in range(3)]
+    ora.active_step(st, ora.GxpoCfg(K=5, alpha=0.5), lambda w, th: gs[w])
+    assert st.t_opt == 3
+    # moments are those of three plain AdamW updates with g0, g1, g_slow (never rewound)
+    m = np.zeros(n)
+    v = np.zeros(n)
+    for g in gs:
+        m = 0.9 * m + (1 - 0.9) * g
+        v = 0.999 * v + (1 - 0.999) * g * g
+    np.testing.assert_allclose(st.m, m, rtol=1e-13)
+    np.testing.assert_allclose(st.v, v, rtol=1e-13)
+
+
+# ---------------------------------------------------------------------------
+# norm
+# ---------------------------------------------------------------------------
+def test_norm_closed_forms_and_library():
+    assert ora.l2norm(np.array([3.0, 4.0])) == 5.0
+    n, c = 10000, -0.37
+    assert ora.l2norm(np.full(n, c)) == pytest.approx(abs(c) * math.sqrt(n), rel=1e-13)
+    x = np.random.default_rng(9).standard_normal(100003)
+    assert ora.l2norm(x) == pytest.approx(float(np.linalg.norm(x)), rel=1e-13)
+    assert ora.l2norm(8.0 * x) == pytest.approx(8.0 * ora.l2norm(x), rel=1e-15)
+    assert ora.l2norm(np.zeros(0)) == 0.0
+
+
+def test_bf16_conversion_helpers_are_exact():
+    x = np.array([1.0, -2.5, 3.140625, 1e-3, 0.0, -0.0, 65504.0], dtype=np.float32)
+    bits = workloads.f32_to_bf16_bits(x)
+    back = workloads.bf16_bits_to_f32(bits)
+    # bf16 keeps 8 significand bits: relative error <= 2^-9, and the round trip is idempotent
+    assert np.all(np.abs(back - x) <= np.abs(x) * 2.0**-8)
+    np.testing.assert_array_equal(workloads.f32_to_bf16_bits(back), bits)
+    np.testing.assert_array_equal(ora.bf16_bits_to_f64(bits), back.astype(np.float64))
+    # ties go to even: 1 + 2^-8 is halfway between 1 and 1 + 2^-7
+    tie = np.array([1.0 + 2.0**-8, 1.0 + 3 * 2.0**-8], dtype=np.float32)
+    np.testing.assert_array_equal(workloads.bf16_bits_to_f32(workloads.f32_to_bf16_bits(tie)),
+                                  np.array([1.0, 1.0 + 2.0**-6], dtype=np.float32))
