@@ -1,0 +1,415 @@
+#!/usr/bin/env python
+"""Benchmark of the GXPO active step on B200.
+
+A "step" is one whole active step of Algorithm 1's parameter-space update over
+the workload's tensor list: probe step 0, probe step 1, extrapolate + reposition,
+slow step with the in-sweep norm, gate update (4 sweeps + 1 tiny kernel).  The
+three gradient buffers are synthetic and already resident.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "GXPO active-step params/sec"
+UNIT = "params/s"
+BYTES_STEP_ADAMW = 26      # R theta, m, v (12) + g bf16 (2); W theta, m, v (12)
+BYTES_EXTRAP = 16          # R theta2, theta0 (8) + g0, g1 bf16 (4); W theta-tilde (4)
+BYTES_ACTIVE = {0: 94, 1: 98}   # per placement: PINGPONG, SNAPSHOT (+4: theta^t copy)
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="qwen25_7b",
+                    choices=["qwen25_7b", "llama31_8b", "flat_1p54b", "small"])
+    ap.add_argument("--layers", type=int, default=0, help="override the decoder depth (0 = full)")
+    ap.add_argument("--K", type=int, default=5)
+    ap.add_argument("--alpha", type=float, default=0.5)
+    ap.add_argument("--lr", type=float, default=1e-7)
+    ap.add_argument("--placement", type=int, default=0)
+    ap.add_argument("--variant", type=int, default=0)
+    ap.add_argument("--ctas", type=int, default=0)
+    ap.add_argument("--fallback", action="store_true", help="time the single-pass fallback step")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-params", type=int, default=1 << 26)
+    ap.add_argument("--cpu-params", type=int, default=1 << 24)
+    return ap.parse_args()
+
+
+def workload_shapes(args):
+    from paper_2605_06755_b200 import workloads as w
+    if args.workload == "qwen25_7b":
+        return w.qwen25_7b_shapes(args.layers or 28), "Qwen2.5-7B-shaped tensor list"
+    if args.workload == "llama31_8b":
+        return w.llama31_8b_shapes(args.layers or 32), "Llama-3.1-8B-shaped tensor list"
+    if args.workload == "flat_1p54b":
+        return [("flat", w.FLAT_QWEN25_1P5B)], "flat 1.54e9-parameter buffer"
+    return w.qwen25_7b_shapes(args.layers or 1), "Qwen2.5-7B-shaped list, reduced depth"
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def recorded_traffic_per_param():
+    """DRAM bytes per parameter of the dominant kernel from the committed ncu summary."""
+    path = os.path.join(ROOT, "profiles", "step_kernel_traffic.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["dram_bytes_per_param"])
+    except Exception:
+        return None
+
+
+# ----------------------------------------------------------------------------
+# clocks
+# ----------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("uuid,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+
+    def __init__(self, uuid: str):
+        self.uuid = uuid
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) == 8:
+                self.rows.append((time.time(), parts))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        mine = [p for (ts, p) in self.rows if (self.uuid in p[0] or not self.uuid) and t0 - 0.05 <= ts <= t1 + 0.15]
+        if not mine:
+            mine = [p for (ts, p) in self.rows if self.uuid in p[0] or not self.uuid]
+        sm = [float(p[1]) for p in mine if p[1].replace(".", "").isdigit()]
+        mx = [float(p[2]) for p in mine if p[2].replace(".", "").isdigit()]
+        pw = [float(p[3]) for p in mine if p[3].replace(".", "").isdigit()]
+        reasons = [n for i, n in enumerate(self.NAMES) if any(p[4 + i].lower().startswith("active") for p in mine)]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None, "reasons": reasons, "samples": len(mine)}
+
+
+# ----------------------------------------------------------------------------
+# CPU oracle legs
+# ----------------------------------------------------------------------------
+def oracle_sample(n, seed, K, alpha, lr):
+    """Inputs of one active step on an n-parameter slice, as the oracle's float64 arrays."""
+    import numpy as np
+    from oracle import gxpo_oracle as ora
+    from paper_2605_06755_b200 import workloads as w
+    th, m, v, g0, g1, gs = w.llm_inputs_numpy(n, seed, "bf16")
+    grads = [ora.bf16_bits_to_f64(g) for g in (g0, g1, gs)]
+    opt = ora.OptCfg(kind="adamw", lr=float(np.float32(lr)), beta1=float(np.float32(0.9)),
+                     beta2=float(np.float32(0.999)), eps=float(np.float32(1e-8)),
+                     weight_decay=float(np.float32(0.01)))
+    cfg = ora.GxpoCfg(K=K, alpha=alpha, delta=float(np.float32(1e-8)))
+    st = ora.State(th, opt, m, v)
+    return ora, st, cfg, grads
+
+
+def time_oracle_steps(n, K, alpha, lr, steps, warmup, min_seconds=0.0):
+    ora, st, cfg, grads = oracle_sample(n, 1234, K, alpha, lr)
+    gate = ora.Gate(cfg)
+    fn = lambda which, theta: grads[which]
+    import numpy as np
+    with np.errstate(all="ignore"):
+        for _ in range(warmup):
+            ora.train_step(st, gate, cfg, fn, round_f32=True)
+        done, t0 = 0, time.perf_counter()
+        while done < steps or (time.perf_counter() - t0) < min_seconds:
+            ora.train_step(st, gate, cfg, fn, round_f32=True)
+            done += 1
+        dt = time.perf_counter() - t0
+    return done, dt
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    shapes, desc = workload_shapes(args)
+    n = args.cpu_params
+    done, dt = time_oracle_steps(n, args.K, args.alpha, args.lr, args.steps, args.warmup)
+    value = n * done / dt
+    sample = (f"{n}-parameter slice drawn with the workload's recipe, one oracle active step "
+              f"(double arithmetic, fp32 rounding between calls) per bench step")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": done, "warmup": args.warmup, "ms_per_step": 1e3 * dt / done, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": desc, "params": sum(k for _, k in shapes), "tensors": len(shapes),
+                   "optimizer": "AdamW", "K": args.K, "alpha": args.alpha, "lr": args.lr, "grad_dtype": "bf16"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------
+# the CUDA path
+# ----------------------------------------------------------------------------
+def build_device_workload(torch, b, shapes, seed, alias_gslow):
+    from paper_2605_06755_b200 import workloads as w
+    d = sum(k for _, k in shapes)
+    dev = torch.device("cuda", torch.cuda.current_device())
+    theta = torch.empty(d, dtype=torch.float32, device=dev)
+    work = torch.empty(d, dtype=torch.float32, device=dev)
+    m = torch.empty(d, dtype=torch.float32, device=dev)
+    v = torch.empty(d, dtype=torch.float32, device=dev)
+    g0 = torch.empty(d, dtype=torch.bfloat16, device=dev)
+    g1 = torch.empty(d, dtype=torch.bfloat16, device=dev)
+    gs = g0 if alias_gslow else torch.empty(d, dtype=torch.bfloat16, device=dev)
+    w.fill_llm_inputs_torch(theta, m, v, g0, g1, None if alias_gslow else gs, seed)
+    work.zero_()
+    ptrs, off = [], 0
+    for _, k in shapes:
+        ptrs.append(b.TensorPtrs(theta.data_ptr() + 4 * off, work.data_ptr() + 4 * off,
+                                 m.data_ptr() + 4 * off, v.data_ptr() + 4 * off,
+                                 g0.data_ptr() + 2 * off, g1.data_ptr() + 2 * off,
+                                 gs.data_ptr() + 2 * off, k))
+        off += k
+    return d, ptrs, (theta, work, m, v, g0, g1, gs)
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2605_06755_b200 import build
+    build.build_library()
+    from paper_2605_06755_b200 import binding as b
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA library is the only compute path")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    props = torch.cuda.get_device_properties(local)
+    stream = torch.cuda.current_stream()
+
+    shapes, desc = workload_shapes(args)
+    d = sum(k for _, k in shapes)
+    free, total = torch.cuda.mem_get_info()
+    margin = 6 << 30
+    alias = False
+    if 22 * d + margin > free:
+        alias = True                      # g_slow reuses g0's buffer (g0 is dead after extrapolate)
+    while (20 if alias else 22) * d + margin > free and args.workload in ("qwen25_7b", "llama31_8b"):
+        args.layers = (args.layers or (28 if args.workload == "qwen25_7b" else 32)) - 1
+        shapes, desc = workload_shapes(args)
+        desc += f" (reduced to {args.layers} layers: not enough free device memory)"
+        d = sum(k for _, k in shapes)
+    d, ptrs, keep = build_device_workload(torch, b, shapes, 1000 + rank, alias)
+    sumsq = torch.zeros(1, dtype=torch.float64, device="cuda")
+
+    cfg, opt = b.make_cfg(K=args.K, alpha=args.alpha, lr=args.lr, placement=args.placement)
+    ctx = b.Context(cfg, opt, b.BF16)
+    ctx.tune(args.ctas, args.variant)
+    ctx.bind(ptrs)
+    if world > 1:
+        ctx.set_sumsq_buffer(sumsq.data_ptr())
+
+    n_ev = 5
+    def one_step(evs=None):
+        if args.fallback:
+            if evs: evs[0].record(stream)
+            ctx.probe_step(-1, stream)
+            if evs: evs[1].record(stream)
+            return None
+        if evs: evs[0].record(stream)
+        ctx.probe_step(0, stream)
+        if evs: evs[1].record(stream)
+        ctx.probe_step(1, stream)
+        if evs: evs[2].record(stream)
+        ctx.extrapolate(stream)
+        if evs: evs[3].record(stream)
+        ctx.slow_step(stream)
+        if evs: evs[4].record(stream)
+        if world > 1:
+            dist.all_reduce(sumsq)        # the one exchange of a sharded step: 8 bytes
+        return ctx.gate_update(stream, allow_nonfinite=True)
+
+    for _ in range(max(args.warmup, 3)):
+        one_step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(n_ev)] for _ in range(args.steps)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(str(getattr(props, "uuid", "")))
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    launches0 = ctx.launch_count()
+    torch.cuda.synchronize()
+    t_wall0 = time.time()
+    e0.record(stream)
+    res = None
+    for s in range(args.steps):
+        res = one_step(evs[s])
+    e1.record(stream)
+    torch.cuda.synchronize()
+    t_wall1 = time.time()
+    if world > 1:
+        dist.barrier()
+    launches = ctx.launch_count() - launches0
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    ms_total = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+
+    # per-kernel durations from the events inside the timed region
+    names = ["probe_step0", "probe_step1", "extrapolate", "slow_step"]
+    per = {}
+    if not args.fallback:
+        for i, nm in enumerate(names):
+            per[nm] = statistics.mean(evs[s][i].elapsed_time(evs[s][i + 1]) for s in range(args.steps))
+        step_ms = statistics.mean([per["probe_step0"], per["probe_step1"], per["slow_step"]])
+    else:
+        per["fallback_step"] = statistics.mean(evs[s][0].elapsed_time(evs[s][1]) for s in range(args.steps))
+        step_ms = per["fallback_step"]
+
+    peak, peak_kind = measured_peak_gbs()
+    bytes_probe0 = BYTES_STEP_ADAMW + (4 if args.placement == 1 else 0)
+    alg_bytes = {"probe_step0": bytes_probe0, "probe_step1": BYTES_STEP_ADAMW, "extrapolate": BYTES_EXTRAP,
+                 "slow_step": BYTES_STEP_ADAMW, "fallback_step": BYTES_STEP_ADAMW}
+    kernels = {nm: {"ms": ms, "gbs": alg_bytes[nm] * d / (ms * 1e-3) / 1e9} for nm, ms in per.items()}
+    achieved = BYTES_STEP_ADAMW * d / (step_ms * 1e-3) / 1e9 if args.placement == 0 or args.fallback else \
+        statistics.mean([kernels["probe_step1"]["gbs"], kernels["slow_step"]["gbs"]])
+    tpp = recorded_traffic_per_param()
+    roofline = {"bound": "hbm", "kernel": "step_kernel (AdamW sweep: probe steps, slow step, fallback)",
+                "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "peak_kind": f"of {peak_kind}", "traffic": (tpp * d if tpp else None),
+                "algorithmic_bytes_per_launch": BYTES_STEP_ADAMW * d}
+    step_bytes = (BYTES_STEP_ADAMW if args.fallback else BYTES_ACTIVE[args.placement]) * d
+    whole_gbs = step_bytes / (ms_step * 1e-3) / 1e9
+
+    total_params = d * world
+    line = {
+        "metric": METRIC, "value": total_params / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": desc, "params_per_gpu": d, "tensors": len(shapes), "optimizer": "AdamW",
+                   "K": args.K, "alpha": args.alpha, "lr": args.lr, "grad_dtype": "bf16",
+                   "placement": ["pingpong", "snapshot"][args.placement],
+                   "step": "fallback (single pass)" if args.fallback else "active (probe, probe, extrapolate, slow step, gate)",
+                   "g_slow_aliases_g0": alias, "l2": "inputs larger than L2 (no flush needed)",
+                   "parallelism": f"dp{world} (independent shards, one 8-byte all-reduce per step)" if world > 1 else "1 GPU"},
+        "hbm_gbs_whole_step": whole_gbs, "hbm_frac_whole_step": whole_gbs / peak,
+        "hbm_frac_of_8tbs_nominal": whole_gbs / 8000.0,
+        "bytes_per_param_per_step": step_bytes / d,
+        "kernels": kernels, "roofline": roofline, "clocks": clocks, "gpu_launches": launches,
+        "gate": None if res is None else {"norm": res.norm, "t": res.t, "active": res.active},
+    }
+
+    if rank == 0 and not args.no_e2e:
+        line["e2e"] = run_e2e(torch, b, args, cfg, opt)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        n = args.cpu_params
+        done, dt = time_oracle_steps(n, args.K, args.alpha, args.lr, 2, 1, min_seconds=10.0)
+        line["cpu_baseline"] = {
+            "value": n * done / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"{done} oracle active steps on a {n}-parameter slice drawn with the workload's recipe "
+                      f"({dt:.1f} s on one of {os.cpu_count()} host cores)"}
+    ctx.close()
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_e2e(torch, b, args, cfg, opt):
+    """The same step through gxpo_step_host: parameters, optimizer state and the
+    three gradients start in pinned HOST memory; results are copied back."""
+    n = args.e2e_params
+    from paper_2605_06755_b200 import workloads as w
+    import numpy as np
+    th, m, v, g0, g1, gs = w.llm_inputs_numpy(n, 4321, "bf16")
+    pin = [torch.from_numpy(x.view(np.int16) if x.dtype == np.uint16 else x).pin_memory()
+           for x in (th, m, v, g0, g1, gs)]
+    ctx = b.Context(cfg, opt, b.BF16)
+    ctx.tune(args.ctas, args.variant)
+    t = [b.tensor_ptrs(pin[0], None, pin[1], pin[2], pin[3], pin[4], pin[5])]
+    l0 = None
+    for i in range(2 + 3):
+        if i == 2:
+            torch.cuda.synchronize()
+            l0 = ctx.launch_count()
+            t0 = time.perf_counter()
+        ctx.step_host(t, staging_elems=1 << 23, allow_nonfinite=True)
+    torch.cuda.synchronize()
+    dt = (time.perf_counter() - t0) / 3
+    launches = (ctx.launch_count() - l0) // 3
+    ctx.close()
+    return {"value": n / dt, "unit": UNIT, "h2d_bytes_per_step": 18 * n, "d2h_bytes_per_step": 12 * n + 64,
+            "ms_per_step": dt * 1e3, "gpu_launches_per_step": launches,
+            "sample": f"{n}-parameter flat slice; theta, m, v, g0, g1, g_slow in pinned host memory, "
+                      f"streamed through gxpo_step_host in 8388608-parameter pieces"}
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

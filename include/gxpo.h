@@ -1,0 +1,238 @@
+/*
+ * gxpo.h -- C ABI of the GXPO active-phase parameter update for NVIDIA B200 (sm_100a).
+ *
+ * GXPO (Gradient Extrapolation-Based Policy Optimization) replaces one optimizer
+ * step of a GRPO trainer by: two fast probe optimizer steps, a per-coordinate
+ * geometric extrapolation of the observed two-step displacement to a virtual
+ * K-step point, a partial move towards it, one corrective optimizer step with the
+ * gradient taken at the repositioned point, and a rolling z-score gate on the norm
+ * of that gradient which permanently falls back to the single-pass step
+ * (Algorithm 1 of the paper).  This library is the parameter-space part of that
+ * step.  The three backward passes stay with the caller: gradients come in as
+ * device buffers.
+ *
+ * Conventions
+ *   - Every pointer inside gxpo_tensor is a DEVICE pointer owned by the caller; the
+ *     library never allocates, frees or keeps parameter memory.  Pointers passed to
+ *     the *_host entry points are HOST pointers (see there).
+ *   - theta, work, m, v are float32.  Gradients are float32 or bfloat16, one dtype
+ *     per context.  Arithmetic is float32; the norm is accumulated in float64.
+ *   - Every call returns a gxpo_status; nothing throws, aborts or traps.  The text
+ *     of the last failure is available from gxpo_last_error().
+ *   - Sweeps are asynchronous on the cudaStream_t passed as `stream` (void*, may be
+ *     NULL for the legacy default stream).  Only gxpo_gate_update and
+ *     gxpo_state_export wait for the device.
+ *   - Vector (128/256-bit) access is used for a tensor when all of its bound
+ *     pointers are 32-byte aligned; otherwise that tensor takes a slower scalar
+ *     path with identical results.  Any n >= 0 is accepted; n == 0 is a no-op.
+ *   - A context is not thread-safe; use one per host thread or lock around it.
+ *   - One GPU per context: the device current at gxpo_create.
+ */
+#ifndef GXPO_H
+#define GXPO_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct gxpo_ctx gxpo_ctx; /* opaque, library-owned */
+
+typedef enum {
+    GXPO_OK = 0,
+    GXPO_ERR_INVALID_ARG = 1, /* null pointer, negative size, K < 2, alpha outside [0,1], ... */
+    GXPO_ERR_ALIGNMENT = 2,   /* a pointer is not aligned to its element size */
+    GXPO_ERR_STATE = 3,       /* call out of order for Algorithm 1, or nothing bound */
+    GXPO_ERR_CUDA = 4,        /* a CUDA runtime call failed; see gxpo_last_error */
+    GXPO_ERR_TIMEOUT = 5,     /* a bounded device-side wait gave up */
+    GXPO_ERR_NONFINITE = 6    /* ||g_slow|| was not finite; the gate was tripped */
+} gxpo_status;
+
+enum { GXPO_OPT_GD = 0, GXPO_OPT_ADAMW = 1 };  /* base optimizer, "OptimStep" in Algorithm 1 */
+enum { GXPO_F32 = 0, GXPO_BF16 = 1 };          /* gradient dtype */
+
+/* Where the intermediate points live (the paper is silent; both keep theta^t alive
+ * until the extrapolation, as Algorithm 1 needs):
+ *   PINGPONG : probe 0 writes theta^{t,1} into `work`, probe 1 updates `work` in
+ *              place, extrapolate writes theta-tilde into `theta`, the slow step
+ *              updates `theta` in place.  The caller's backward pass 2 reads `work`,
+ *              backward pass 3 reads `theta`.  26+26+16+26 bytes per parameter.
+ *   SNAPSHOT : probe 0 copies theta^t into `work` and writes theta^{t,1} into
+ *              `theta`; every later point is written into `theta`, so a model that
+ *              aliases `theta` never has to be re-pointed.  30+26+16+26 bytes. */
+enum { GXPO_PLACE_PINGPONG = 0, GXPO_PLACE_SNAPSHOT = 1 };
+
+/* Base optimizer.  GD: theta <- theta - lr g (the paper's surrogate, Sec. 2.1).
+ * AdamW (the paper's experiments; decoupled decay, bias-corrected, constant lr):
+ *   m <- b1 m + (1-b1) g;  v <- b2 v + (1-b2) g^2;
+ *   theta <- theta (1 - lr wd) - lr (m / (1-b1^t)) / (sqrt(v / (1-b2^t)) + eps).
+ * The step count t advances on EVERY optimizer step, probes included (Sec. 2.3). */
+typedef struct {
+    int kind; /* GXPO_OPT_GD or GXPO_OPT_ADAMW */
+    float lr, beta1, beta2, eps, weight_decay;
+} gxpo_opt_cfg;
+
+/* Hyper-parameters of Algorithm 1 ("Require" line) and of the adaptive rule.
+ *   K >= 2 virtual depth, alpha in [0,1] move fraction, delta >= 0 active-set
+ *   threshold (|g0_i| > delta, strict).  den_eps: 0 = the literal scale factor of
+ *   Eq. (scale_factor); > 0 = coordinates with |1 + r_i| <= den_eps keep scale 1.
+ *   tau, gate_eps, window: Eq. (z_score).  min_history: the z-score is evaluated
+ *   once the buffer holds at least this many norms (Algorithm 1: 2).  std_ddof: 0
+ *   population, 1 sample standard deviation. */
+typedef struct {
+    int K;
+    float alpha, delta, den_eps;
+    double tau, gate_eps;
+    int window, min_history, std_ddof;
+    int placement; /* GXPO_PLACE_* */
+} gxpo_cfg;
+
+/* One parameter tensor.  `work` has the same length as `theta`.  m and v may be
+ * NULL for GXPO_OPT_GD.  g0/g1/g_slow are read-only inputs of the context's
+ * gradient dtype; g_slow may alias g0 or g1 (both are dead once gxpo_extrapolate
+ * has run).  No other buffers may overlap. */
+typedef struct {
+    float* theta;
+    float* work;
+    float* m;
+    float* v;
+    const void* g0;
+    const void* g1;
+    const void* g_slow;
+    long long n;
+} gxpo_tensor;
+
+/* What the gate saw at the end of an active step (Eq. (z_score)). z, mu, sigma are
+ * NaN while the buffer is still warming up. */
+typedef struct {
+    int active;        /* 1 if the NEXT step is still an active step (t < s_star) */
+    int tripped;       /* 1 if this update set s_star */
+    long long t;       /* index of the next training step */
+    long long s_star;  /* first fallback step, -1 while unset */
+    double norm, z, mu, sigma;
+} gxpo_gate_result;
+
+/* Fill cfg/opt with the values the paper's experiments state (K=5, alpha=0.5,
+ * delta=1e-8, tau=0.5, lr=1e-7) and this library's documented choices for what the
+ * paper leaves open (AdamW betas 0.9/0.999, eps 1e-8, weight decay 0.01; window 20,
+ * gate_eps 1e-8, min_history 2, population std, den_eps 0, PINGPONG). */
+void gxpo_default_cfg(gxpo_cfg* cfg, gxpo_opt_cfg* opt);
+
+/* Create a context on the current device.  Allocates a few KB of device scratch
+ * (partial sums, gate ring buffer) and one pinned result slot.
+ * Errors: INVALID_ARG for bad hyper-parameters, CUDA if allocation fails. */
+gxpo_status gxpo_create(const gxpo_cfg* cfg, const gxpo_opt_cfg* opt, int grad_dtype,
+                        gxpo_ctx** out);
+void gxpo_destroy(gxpo_ctx* ctx);
+
+/* Bind a tensor list (count == 1 is the flat-buffer case).  Copies the descriptors
+ * and builds the chunk table on the device; the list itself is not kept.  May be
+ * called again between steps to re-bind.  Waits for the device before it replaces
+ * an earlier table.
+ * Errors: INVALID_ARG (null list entry fields, n < 0, count < 0, m/v missing for
+ * AdamW), ALIGNMENT (pointer not aligned to its element size), STATE (mid-step). */
+gxpo_status gxpo_bind(gxpo_ctx* ctx, const gxpo_tensor* list, int count);
+
+/* Algorithm 1, "first/second fast optimizer step" (which = 0, 1) and the fallback
+ * phase's single step (which = -1).
+ *   which =  0: theta^{t,1} <- OptimStep(theta^t, g0)      state: IDLE   -> PROBED0
+ *               illegal once the gate has tripped (t >= s_star).
+ *   which =  1: theta^{t,2} <- OptimStep(theta^{t,1}, g1)  state: PROBED0 -> PROBED1
+ *   which = -1: theta^{t+1} <- OptimStep(theta^t, g0) in place in `theta`, the
+ *               single-pass step Algorithm 1 takes when t >= s_star; legal between
+ *               steps at any time (a caller may also warm up with it); advances t.
+ * Errors: STATE when called out of order or in the wrong phase. */
+gxpo_status gxpo_probe_step(gxpo_ctx* ctx, int which, void* stream);
+
+/* Algorithm 1, active set through reposition (Eqs. (retention), (scale_factor),
+ * (k_step_position), (blend_step)): per coordinate
+ *   scale = S_K(r)/S_2(r) with r = g1/g0 if |g0| > delta, else 1
+ *   theta-tilde = theta^t + alpha (theta^{t,2} - theta^t) scale      -> `theta`
+ * state: PROBED1 -> EXTRAPOLATED. */
+gxpo_status gxpo_extrapolate(gxpo_ctx* ctx, void* stream);
+
+/* Algorithm 1, "slow correction": theta^{t+1} <- OptimStep(theta-tilde, g_slow), in
+ * place in `theta`, and sum(g_slow^2) accumulated in the same sweep (float64,
+ * deterministic for a fixed launch shape).  state: EXTRAPOLATED -> SLOW_DONE. */
+gxpo_status gxpo_slow_step(gxpo_ctx* ctx, void* stream);
+
+/* Adaptive rule (Eq. (z_score); Algorithm 1 after the slow correction), evaluated
+ * by a device kernel: ||g_slow||, mu and sigma of the stored norms, Z, Z >= tau =>
+ * s_star = t + 1; the norm is pushed either way; t advances.  Waits for `stream`
+ * (one 64-byte read-back).  `out` may be NULL.  state: SLOW_DONE -> IDLE.
+ * Returns NONFINITE (after completing the update and tripping the gate) when the
+ * norm is Inf/NaN -- that rule is this library's, not the paper's. */
+gxpo_status gxpo_gate_update(gxpo_ctx* ctx, void* stream, gxpo_gate_result* out);
+
+/* Sharded parameter sets (one process per GPU, each holding a slice of every
+ * tensor or a subset of the list): the only cross-shard quantity of the whole
+ * update is sum(g_slow^2).  Point the context at a caller-owned DEVICE double;
+ * gxpo_slow_step then writes this shard's sum there and gxpo_gate_update reads
+ * the norm from it, so the caller can sum it across ranks in between (one 8-byte
+ * all-reduce on the same stream).  NULL restores the internal scalar.  With the
+ * same reduced value on every rank the gates flip together. */
+gxpo_status gxpo_set_sumsq_buffer(gxpo_ctx* ctx, double* sumsq_dev);
+
+/* Host-side view of the gate, no device work. */
+gxpo_status gxpo_gate_peek(const gxpo_ctx* ctx, int* active, long long* s_star, long long* t);
+
+/* Optimizer step count so far (3 per active step, 1 per fallback step). */
+long long gxpo_optimizer_steps(const gxpo_ctx* ctx);
+
+/* Backward passes spent so far: 3 s + (t - s) with s = min(s_star, t) (Sec. 2.3). */
+long long gxpo_backward_passes(const gxpo_ctx* ctx);
+
+/* Checkpointing of the small state (gate ring buffer, t, s_star, optimizer step
+ * count).  Call with buf == NULL to get the size in *len.  theta/m/v are the
+ * caller's tensors and are checkpointed by the caller.  Only legal between steps. */
+gxpo_status gxpo_state_export(gxpo_ctx* ctx, void* buf, size_t* len);
+gxpo_status gxpo_state_import(gxpo_ctx* ctx, const void* buf, size_t len);
+
+/* One whole training step of Algorithm 1 for parameters and optimizer state that
+ * live in HOST memory (offloaded optimizer state).  All pointers in `list` are HOST
+ * pointers (pinned memory makes the copies asynchronous); `work` is ignored.  The
+ * three gradients are supplied up front, so this entry point fits callers that
+ * replay stored gradients or whose loss has a closed-form gradient; it streams
+ * pieces of each tensor through device staging buffers owned by the context
+ * (allocated on first use, `staging_elems` parameters per piece), runs the same
+ * kernels on them, and writes theta, m, v back.  If the gate is active it runs an
+ * active step including gxpo_gate_update, otherwise a fallback step with g0.
+ * Does not need gxpo_bind.  Waits for completion. */
+gxpo_status gxpo_step_host(gxpo_ctx* ctx, const gxpo_tensor* list, int count,
+                           long long staging_elems, void* stream, gxpo_gate_result* out);
+
+/* Launch-shape knobs, for benchmarking: resident CTAs per SM (0 = default) and the
+ * memory-access variant (0 = default, 1 = 128-bit loads, 2 = 256-bit loads,
+ * 3 = bulk-copy shared-memory ring).  Results are identical across variants except
+ * for the summation order of the norm. */
+gxpo_status gxpo_tune(gxpo_ctx* ctx, int ctas_per_sm, int variant);
+
+/* Number of kernels this context has launched so far. */
+long long gxpo_launch_count(const gxpo_ctx* ctx);
+
+const char* gxpo_last_error(const gxpo_ctx* ctx);
+const char* gxpo_status_string(gxpo_status s);
+
+/* ---- Surrogate harness (the paper's diagonal-quadratic sanity check, Corollary 1):
+ *      f(theta) = sum_i a_i theta_i^2 / 2 - b_i theta_i.  Not part of the update; it
+ *      stands in for the caller's backward pass in tests and benchmarks. ---------- */
+
+/* g <- a * theta - b, float32, rounded after the product and after the difference. */
+gxpo_status gxpo_quad_grad(const float* theta, const float* a, const float* b, float* g,
+                           long long n, void* stream);
+
+/* One whole active step with plain GD on the surrogate in a single sweep: the three
+ * gradients are recomputed in registers.  theta is updated in place; sum(g_slow^2)
+ * is written to *sumsq_dev (device pointer to one double).  16 bytes per parameter.
+ * `scratch_dev` is gxpo_quad_scratch_bytes() of device memory that the caller
+ * zeroes once before the first call and then leaves alone. */
+gxpo_status gxpo_quad_active_step(float* theta, const float* a, const float* b, long long n,
+                                  float lr, int K, float alpha, float delta, float den_eps,
+                                  double* sumsq_dev, void* scratch_dev, void* stream);
+size_t gxpo_quad_scratch_bytes(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GXPO_H */

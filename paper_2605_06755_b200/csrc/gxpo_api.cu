@@ -1,0 +1,706 @@
+// Host side of the GXPO library: context, argument checks, the call-order state
+// machine of Algorithm 1, chunk tables and kernel launches.  C ABI in include/gxpo.h.
+#include "gxpo.h"
+#include "gxpo_kernels.cuh"
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+using namespace gxpo;
+
+namespace {
+
+enum Phase { IDLE = 0, PROBED0 = 1, PROBED1 = 2, EXTRAPOLATED = 3, SLOW_DONE = 4 };
+
+struct Staging {                       // device pieces for gxpo_step_host
+    long long elems = 0;
+    int slots = 0;
+    float* theta[3] = {nullptr, nullptr, nullptr};
+    float* work[3] = {nullptr, nullptr, nullptr};
+    float* m[3] = {nullptr, nullptr, nullptr};
+    float* v[3] = {nullptr, nullptr, nullptr};
+    void* g[3][3] = {{nullptr, nullptr, nullptr}, {nullptr, nullptr, nullptr}, {nullptr, nullptr, nullptr}};
+    cudaStream_t stream[3] = {nullptr, nullptr, nullptr};
+    cudaEvent_t done[3] = {nullptr, nullptr, nullptr};
+    double* piece_sumsq = nullptr;     // device accumulator across pieces
+};
+
+}  // namespace
+
+struct gxpo_ctx {
+    gxpo_cfg cfg;
+    gxpo_opt_cfg opt;
+    int grad_dtype;
+    int device;
+    int sm_count;
+    int ctas_per_sm;                   // 0 = default
+    int variant;                       // 1 = 128-bit, 2 = 256-bit
+    Phase phase;
+    // bound list
+    TensorDesc* d_descs;
+    ChunkRef* d_chunks;
+    long long num_chunks;
+    int num_tensors;
+    int bound;
+    long long total_params;
+    // reductions and gate
+    double* d_partials;
+    unsigned* d_ticket;
+    double* d_sumsq;
+    double* user_sumsq;                // caller-owned replacement for d_sumsq, or null
+    GateState* d_gate;
+    double* d_ring;
+    GateResult* d_result;
+    GateResult* h_result;              // pinned
+    // host mirror
+    long long t, s_star, t_opt;
+    long long launches;
+    Staging stg;
+    char err[512];
+};
+
+namespace {
+
+gxpo_status fail(gxpo_ctx* c, gxpo_status s, const char* fmt, ...) {
+    if (c) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(c->err, sizeof(c->err), fmt, ap);
+        va_end(ap);
+    }
+    return s;
+}
+
+#define CUDA_TRY(c, call)                                                                 \
+    do {                                                                                  \
+        cudaError_t e_ = (call);                                                          \
+        if (e_ != cudaSuccess)                                                            \
+            return fail((c), GXPO_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_)); \
+    } while (0)
+
+bool finite_f(float x) { return std::isfinite(x); }
+
+gxpo_status check_cfg(gxpo_ctx* c, const gxpo_cfg* g, const gxpo_opt_cfg* o, int grad_dtype) {
+    if (g->K < 2 || g->K > 4096) return fail(c, GXPO_ERR_INVALID_ARG, "K must be in [2, 4096], got %d", g->K);
+    if (!(g->alpha >= 0.0f && g->alpha <= 1.0f)) return fail(c, GXPO_ERR_INVALID_ARG, "alpha must be in [0, 1]");
+    if (!(g->delta >= 0.0f) || !finite_f(g->delta)) return fail(c, GXPO_ERR_INVALID_ARG, "delta must be finite and >= 0");
+    if (!(g->den_eps >= 0.0f) || !finite_f(g->den_eps)) return fail(c, GXPO_ERR_INVALID_ARG, "den_eps must be finite and >= 0");
+    if (std::isnan(g->tau)) return fail(c, GXPO_ERR_INVALID_ARG, "tau is NaN");
+    if (!(g->gate_eps >= 0.0)) return fail(c, GXPO_ERR_INVALID_ARG, "gate_eps must be >= 0");
+    if (g->window < 1 || g->window > (1 << 20)) return fail(c, GXPO_ERR_INVALID_ARG, "window must be in [1, 2^20]");
+    if (g->min_history < 1) return fail(c, GXPO_ERR_INVALID_ARG, "min_history must be >= 1");
+    if (g->std_ddof < 0 || g->std_ddof > 1) return fail(c, GXPO_ERR_INVALID_ARG, "std_ddof must be 0 or 1");
+    if (g->placement != GXPO_PLACE_PINGPONG && g->placement != GXPO_PLACE_SNAPSHOT)
+        return fail(c, GXPO_ERR_INVALID_ARG, "unknown placement %d", g->placement);
+    if (o->kind != GXPO_OPT_GD && o->kind != GXPO_OPT_ADAMW) return fail(c, GXPO_ERR_INVALID_ARG, "unknown optimizer kind %d", o->kind);
+    if (!finite_f(o->lr)) return fail(c, GXPO_ERR_INVALID_ARG, "lr is not finite");
+    if (o->kind == GXPO_OPT_ADAMW) {
+        if (!(o->beta1 >= 0.0f && o->beta1 < 1.0f) || !(o->beta2 >= 0.0f && o->beta2 < 1.0f))
+            return fail(c, GXPO_ERR_INVALID_ARG, "betas must be in [0, 1)");
+        if (!(o->eps >= 0.0f) || !finite_f(o->eps)) return fail(c, GXPO_ERR_INVALID_ARG, "eps must be finite and >= 0");
+        if (!finite_f(o->weight_decay)) return fail(c, GXPO_ERR_INVALID_ARG, "weight_decay is not finite");
+    }
+    if (grad_dtype != GXPO_F32 && grad_dtype != GXPO_BF16) return fail(c, GXPO_ERR_INVALID_ARG, "unknown gradient dtype %d", grad_dtype);
+    return GXPO_OK;
+}
+
+int grid_for(const gxpo_ctx* c, long long num_chunks, int default_per_sm) {
+    const int per_sm = c->ctas_per_sm > 0 ? c->ctas_per_sm : default_per_sm;
+    long long g = (long long)c->sm_count * per_sm;
+    if (g > kMaxGrid) g = kMaxGrid;
+    if (g > num_chunks) g = num_chunks;
+    if (g < 1) g = 1;
+    return (int)g;
+}
+
+StepParams make_step_params(gxpo_ctx* c, int which_grad, int in_sel, int out_sel, int snapshot,
+                            int want_norm) {
+    StepParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.which_grad = which_grad;
+    p.in_sel = in_sel;
+    p.out_sel = out_sel;
+    p.snapshot = snapshot;
+    p.want_norm = want_norm;
+    const gxpo_opt_cfg& o = c->opt;
+    p.lr = o.lr;
+    if (o.kind == GXPO_OPT_ADAMW) {
+        // constants are formed in double from the float hyper-parameters, rounded once
+        const double t = (double)c->t_opt;   // already incremented for this step
+        const double b1 = (double)o.beta1, b2 = (double)o.beta2, lr = (double)o.lr;
+        p.beta1 = o.beta1;
+        p.beta2 = o.beta2;
+        p.omb1 = (float)(1.0 - b1);
+        p.omb2 = (float)(1.0 - b2);
+        p.eps = o.eps;
+        p.decay = (float)(1.0 - lr * (double)o.weight_decay);
+        p.step_size = (float)(lr / (1.0 - std::pow(b1, t)));
+        p.inv_sqrt_bc2 = (float)(1.0 / std::sqrt(1.0 - std::pow(b2, t)));
+    }
+    return p;
+}
+
+template <bool ADAMW, typename G>
+void launch_step_t(int variant, int grid, cudaStream_t s, const TensorDesc* descs,
+                   const ChunkRef* chunks, long long num_chunks, const TensorDesc& flat,
+                   const StepParams& p, double* partials, unsigned* ticket, double* sumsq) {
+    if (variant == 1)
+        step_kernel<ADAMW, G, 4><<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, partials, ticket, sumsq);
+    else
+        step_kernel<ADAMW, G, 8><<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, partials, ticket, sumsq);
+}
+
+// Launch one OptimStep sweep over either the bound list (chunks != null) or one
+// flat piece described by `flat`.
+gxpo_status launch_step(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
+                        long long num_chunks, const TensorDesc& flat, const StepParams& p,
+                        double* sumsq) {
+    if (num_chunks <= 0) {
+        if (p.want_norm) CUDA_TRY(c, cudaMemsetAsync(sumsq, 0, sizeof(double), s));
+        return GXPO_OK;
+    }
+    const bool adamw = c->opt.kind == GXPO_OPT_ADAMW;
+    const int grid = grid_for(c, num_chunks, adamw ? 4 : 6);
+    const bool bf16 = c->grad_dtype == GXPO_BF16;
+    if (adamw && bf16) launch_step_t<true, uint16_t>(c->variant, grid, s, descs, chunks, num_chunks, flat, p, c->d_partials, c->d_ticket, sumsq);
+    else if (adamw) launch_step_t<true, float>(c->variant, grid, s, descs, chunks, num_chunks, flat, p, c->d_partials, c->d_ticket, sumsq);
+    else if (bf16) launch_step_t<false, uint16_t>(c->variant, grid, s, descs, chunks, num_chunks, flat, p, c->d_partials, c->d_ticket, sumsq);
+    else launch_step_t<false, float>(c->variant, grid, s, descs, chunks, num_chunks, flat, p, c->d_partials, c->d_ticket, sumsq);
+    c->launches += 1;
+    CUDA_TRY(c, cudaGetLastError());
+    return GXPO_OK;
+}
+
+gxpo_status launch_extrap(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
+                          long long num_chunks, const TensorDesc& flat, const ExtrapParams& p) {
+    if (num_chunks <= 0) return GXPO_OK;
+    const int grid = grid_for(c, num_chunks, 6);
+    const bool bf16 = c->grad_dtype == GXPO_BF16;
+    if (c->variant == 1) {
+        if (bf16) extrap_kernel<uint16_t, 4><<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p);
+        else extrap_kernel<float, 4><<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p);
+    } else {
+        if (bf16) extrap_kernel<uint16_t, 8><<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p);
+        else extrap_kernel<float, 8><<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p);
+    }
+    c->launches += 1;
+    CUDA_TRY(c, cudaGetLastError());
+    return GXPO_OK;
+}
+
+ExtrapParams make_extrap_params(const gxpo_ctx* c, int placement) {
+    ExtrapParams p;
+    p.K = c->cfg.K;
+    p.alpha = c->cfg.alpha;
+    p.delta = c->cfg.delta;
+    p.den_eps = c->cfg.den_eps;
+    if (placement == GXPO_PLACE_PINGPONG) { p.theta2_sel = 1; p.theta0_sel = 0; }
+    else { p.theta2_sel = 0; p.theta0_sel = 1; }
+    return p;
+}
+
+bool gate_active(const gxpo_ctx* c) { return c->s_star < 0 || c->t < c->s_star; }
+
+gxpo_status run_gate(gxpo_ctx* c, cudaStream_t s, const double* sumsq, gxpo_gate_result* out) {
+    gate_kernel<<<1, 32, 0, s>>>(c->d_gate, c->d_ring, sumsq, c->t, c->cfg.tau, c->cfg.gate_eps,
+                                 c->cfg.window, c->cfg.min_history, c->cfg.std_ddof, c->d_result);
+    c->launches += 1;
+    CUDA_TRY(c, cudaGetLastError());
+    CUDA_TRY(c, cudaMemcpyAsync(c->h_result, c->d_result, sizeof(GateResult), cudaMemcpyDeviceToHost, s));
+    CUDA_TRY(c, cudaStreamSynchronize(s));
+    const GateResult r = *c->h_result;
+    c->t = r.t;
+    c->s_star = r.s_star;
+    if (out) {
+        out->active = r.active;
+        out->tripped = r.tripped;
+        out->t = r.t;
+        out->s_star = r.s_star;
+        out->norm = r.norm;
+        out->z = r.z;
+        out->mu = r.mu;
+        out->sigma = r.sigma;
+    }
+    if (!std::isfinite(r.norm))
+        return fail(c, GXPO_ERR_NONFINITE, "||g_slow|| is not finite at step %lld; gate tripped", r.t - 1);
+    return GXPO_OK;
+}
+
+void free_staging(gxpo_ctx* c) {
+    Staging& st = c->stg;
+    for (int i = 0; i < 3; ++i) {
+        cudaFree(st.theta[i]); cudaFree(st.work[i]); cudaFree(st.m[i]); cudaFree(st.v[i]);
+        for (int k = 0; k < 3; ++k) cudaFree(st.g[i][k]);
+        if (st.stream[i]) cudaStreamDestroy(st.stream[i]);
+        if (st.done[i]) cudaEventDestroy(st.done[i]);
+    }
+    cudaFree(st.piece_sumsq);
+    st = Staging();
+}
+
+gxpo_status ensure_staging(gxpo_ctx* c, long long elems) {
+    Staging& st = c->stg;
+    if (st.elems >= elems && st.slots > 0) return GXPO_OK;
+    free_staging(c);
+    const size_t gsz = (c->grad_dtype == GXPO_BF16) ? 2 : 4;
+    const bool adamw = c->opt.kind == GXPO_OPT_ADAMW;
+    for (int i = 0; i < 2; ++i) {
+        CUDA_TRY(c, cudaMalloc(&st.theta[i], elems * sizeof(float)));
+        CUDA_TRY(c, cudaMalloc(&st.work[i], elems * sizeof(float)));
+        if (adamw) {
+            CUDA_TRY(c, cudaMalloc(&st.m[i], elems * sizeof(float)));
+            CUDA_TRY(c, cudaMalloc(&st.v[i], elems * sizeof(float)));
+        }
+        for (int k = 0; k < 3; ++k) CUDA_TRY(c, cudaMalloc(&st.g[i][k], elems * gsz));
+        CUDA_TRY(c, cudaStreamCreateWithFlags(&st.stream[i], cudaStreamNonBlocking));
+        CUDA_TRY(c, cudaEventCreateWithFlags(&st.done[i], cudaEventDisableTiming));
+    }
+    CUDA_TRY(c, cudaMalloc(&st.piece_sumsq, 2 * sizeof(double)));
+    st.elems = elems;
+    st.slots = 2;
+    return GXPO_OK;
+}
+
+__global__ void accumulate_kernel(double* total, const double* piece) {
+    if (threadIdx.x == 0 && blockIdx.x == 0) *total = __dadd_rn(*total, *piece);
+}
+
+}  // namespace
+
+extern "C" {
+
+void gxpo_default_cfg(gxpo_cfg* cfg, gxpo_opt_cfg* opt) {
+    if (cfg) {
+        cfg->K = 5;
+        cfg->alpha = 0.5f;
+        cfg->delta = 1e-8f;
+        cfg->den_eps = 0.0f;
+        cfg->tau = 0.5;
+        cfg->gate_eps = 1e-8;
+        cfg->window = 20;
+        cfg->min_history = 2;
+        cfg->std_ddof = 0;
+        cfg->placement = GXPO_PLACE_PINGPONG;
+    }
+    if (opt) {
+        opt->kind = GXPO_OPT_ADAMW;
+        opt->lr = 1e-7f;
+        opt->beta1 = 0.9f;
+        opt->beta2 = 0.999f;
+        opt->eps = 1e-8f;
+        opt->weight_decay = 0.01f;
+    }
+}
+
+gxpo_status gxpo_create(const gxpo_cfg* cfg, const gxpo_opt_cfg* opt, int grad_dtype, gxpo_ctx** out) {
+    if (!cfg || !opt || !out) return GXPO_ERR_INVALID_ARG;
+    *out = nullptr;
+    gxpo_status s = check_cfg(nullptr, cfg, opt, grad_dtype);
+    if (s != GXPO_OK) return s;
+    gxpo_ctx* c = new (std::nothrow) gxpo_ctx();
+    if (!c) return GXPO_ERR_INVALID_ARG;
+    std::memset(static_cast<void*>(c), 0, sizeof(*c));
+    new (&c->stg) Staging();
+    c->cfg = *cfg;
+    c->opt = *opt;
+    c->grad_dtype = grad_dtype;
+    c->variant = 2;
+    c->s_star = -1;
+    c->phase = IDLE;
+    cudaError_t e = cudaGetDevice(&c->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device);
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_partials, kMaxGrid * sizeof(double));
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_ticket, sizeof(unsigned));
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_sumsq, sizeof(double));
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_gate, sizeof(GateState));
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_ring, (size_t)cfg->window * sizeof(double));
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_result, sizeof(GateResult));
+    if (e == cudaSuccess) e = cudaMallocHost(&c->h_result, sizeof(GateResult));
+    if (e == cudaSuccess) e = cudaMemset(c->d_ticket, 0, sizeof(unsigned));
+    if (e == cudaSuccess) e = cudaMemset(c->d_sumsq, 0, sizeof(double));
+    if (e == cudaSuccess) e = cudaMemset(c->d_ring, 0, (size_t)cfg->window * sizeof(double));
+    if (e == cudaSuccess) {
+        GateState g0;
+        g0.head = 0; g0.count = 0; g0.s_star = -1;
+        e = cudaMemcpy(c->d_gate, &g0, sizeof(g0), cudaMemcpyHostToDevice);
+    }
+    if (e != cudaSuccess) {
+        gxpo_destroy(c);
+        return GXPO_ERR_CUDA;
+    }
+    *out = c;
+    return GXPO_OK;
+}
+
+void gxpo_destroy(gxpo_ctx* c) {
+    if (!c) return;
+    free_staging(c);
+    cudaFree(c->d_descs);
+    cudaFree(c->d_chunks);
+    cudaFree(c->d_partials);
+    cudaFree(c->d_ticket);
+    cudaFree(c->d_sumsq);
+    cudaFree(c->d_gate);
+    cudaFree(c->d_ring);
+    cudaFree(c->d_result);
+    if (c->h_result) cudaFreeHost(c->h_result);
+    delete c;
+}
+
+static gxpo_status check_tensor(gxpo_ctx* c, const gxpo_tensor& t, int i, bool need_work) {
+    if (t.n < 0) return fail(c, GXPO_ERR_INVALID_ARG, "tensor %d: n < 0", i);
+    if (t.n > (long long)kChunk * 0xFFFFFFFFLL) return fail(c, GXPO_ERR_INVALID_ARG, "tensor %d: n too large", i);
+    if (t.n == 0) return GXPO_OK;
+    if (!t.theta || !t.g0 || !t.g1 || !t.g_slow || (need_work && !t.work))
+        return fail(c, GXPO_ERR_INVALID_ARG, "tensor %d: null theta/work/gradient pointer", i);
+    if (c->opt.kind == GXPO_OPT_ADAMW && (!t.m || !t.v))
+        return fail(c, GXPO_ERR_INVALID_ARG, "tensor %d: AdamW needs m and v", i);
+    const uintptr_t gmask = (c->grad_dtype == GXPO_BF16) ? 1u : 3u;
+    if ((((uintptr_t)t.theta) & 3u) || (((uintptr_t)t.work) & 3u) || (((uintptr_t)t.m) & 3u) ||
+        (((uintptr_t)t.v) & 3u) || (((uintptr_t)t.g0) & gmask) || (((uintptr_t)t.g1) & gmask) ||
+        (((uintptr_t)t.g_slow) & gmask))
+        return fail(c, GXPO_ERR_ALIGNMENT, "tensor %d: a pointer is not aligned to its element size", i);
+    return GXPO_OK;
+}
+
+gxpo_status gxpo_bind(gxpo_ctx* c, const gxpo_tensor* list, int count) {
+    if (!c) return GXPO_ERR_INVALID_ARG;
+    if (count < 0 || (count > 0 && !list)) return fail(c, GXPO_ERR_INVALID_ARG, "bad list/count");
+    if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "gxpo_bind in the middle of a step");
+    std::vector<TensorDesc> descs((size_t)count);
+    std::vector<ChunkRef> chunks;
+    long long total = 0;
+    for (int i = 0; i < count; ++i) {
+        gxpo_status s = check_tensor(c, list[i], i, true);
+        if (s != GXPO_OK) return s;
+        TensorDesc& d = descs[(size_t)i];
+        d.theta = list[i].theta; d.work = list[i].work; d.m = list[i].m; d.v = list[i].v;
+        d.g[0] = list[i].g0; d.g[1] = list[i].g1; d.g[2] = list[i].g_slow;
+        d.n = list[i].n;
+        total += d.n;
+    }
+    chunks.reserve((size_t)(total / kChunk + count));
+    for (int i = 0; i < count; ++i) {
+        const long long nc = (descs[(size_t)i].n + kChunk - 1) / kChunk;
+        for (long long k = 0; k < nc; ++k) chunks.push_back(ChunkRef{(unsigned)i, (unsigned)k});
+    }
+    CUDA_TRY(c, cudaDeviceSynchronize());
+    cudaFree(c->d_descs); c->d_descs = nullptr;
+    cudaFree(c->d_chunks); c->d_chunks = nullptr;
+    c->num_chunks = 0; c->num_tensors = 0; c->total_params = 0;
+    if (count > 0) {
+        CUDA_TRY(c, cudaMalloc(&c->d_descs, descs.size() * sizeof(TensorDesc)));
+        CUDA_TRY(c, cudaMemcpy(c->d_descs, descs.data(), descs.size() * sizeof(TensorDesc), cudaMemcpyHostToDevice));
+    }
+    if (!chunks.empty()) {
+        CUDA_TRY(c, cudaMalloc(&c->d_chunks, chunks.size() * sizeof(ChunkRef)));
+        CUDA_TRY(c, cudaMemcpy(c->d_chunks, chunks.data(), chunks.size() * sizeof(ChunkRef), cudaMemcpyHostToDevice));
+    }
+    c->num_chunks = (long long)chunks.size();
+    c->num_tensors = count;
+    c->total_params = total;
+    c->bound = 1;
+    return GXPO_OK;
+}
+
+gxpo_status gxpo_probe_step(gxpo_ctx* c, int which, void* stream) {
+    if (!c) return GXPO_ERR_INVALID_ARG;
+    if (which < -1 || which > 1) return fail(c, GXPO_ERR_INVALID_ARG, "which must be -1, 0 or 1");
+    if (!c->bound) return fail(c, GXPO_ERR_STATE, "nothing bound: call gxpo_bind first");
+    cudaStream_t s = (cudaStream_t)stream;
+    const TensorDesc none = {};
+    const int place = c->cfg.placement;
+    if (which == -1) {
+        if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "fallback step in the middle of an active step");
+        c->t_opt += 1;
+        StepParams p = make_step_params(c, 0, 0, 0, 0, 0);
+        gxpo_status st = launch_step(c, s, c->d_descs, c->d_chunks, c->num_chunks, none, p, c->d_sumsq);
+        if (st != GXPO_OK) { c->t_opt -= 1; return st; }
+        c->t += 1;
+        return GXPO_OK;
+    }
+    if (which == 0) {
+        if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "probe step 0 must start a step");
+        if (!gate_active(c)) return fail(c, GXPO_ERR_STATE, "gate has tripped (s*=%lld, t=%lld): only fallback steps are legal", c->s_star, c->t);
+        c->t_opt += 1;
+        StepParams p = (place == GXPO_PLACE_PINGPONG) ? make_step_params(c, 0, 0, 1, 0, 0)
+                                                      : make_step_params(c, 0, 0, 0, 1, 0);
+        gxpo_status st = launch_step(c, s, c->d_descs, c->d_chunks, c->num_chunks, none, p, c->d_sumsq);
+        if (st != GXPO_OK) { c->t_opt -= 1; return st; }
+        c->phase = PROBED0;
+        return GXPO_OK;
+    }
+    if (c->phase != PROBED0) return fail(c, GXPO_ERR_STATE, "probe step 1 must follow probe step 0");
+    c->t_opt += 1;
+    StepParams p = (place == GXPO_PLACE_PINGPONG) ? make_step_params(c, 1, 1, 1, 0, 0)
+                                                  : make_step_params(c, 1, 0, 0, 0, 0);
+    gxpo_status st = launch_step(c, s, c->d_descs, c->d_chunks, c->num_chunks, none, p, c->d_sumsq);
+    if (st != GXPO_OK) { c->t_opt -= 1; return st; }
+    c->phase = PROBED1;
+    return GXPO_OK;
+}
+
+gxpo_status gxpo_extrapolate(gxpo_ctx* c, void* stream) {
+    if (!c) return GXPO_ERR_INVALID_ARG;
+    if (c->phase != PROBED1) return fail(c, GXPO_ERR_STATE, "extrapolate must follow probe step 1");
+    const TensorDesc none = {};
+    gxpo_status st = launch_extrap(c, (cudaStream_t)stream, c->d_descs, c->d_chunks, c->num_chunks, none,
+                                   make_extrap_params(c, c->cfg.placement));
+    if (st != GXPO_OK) return st;
+    c->phase = EXTRAPOLATED;
+    return GXPO_OK;
+}
+
+gxpo_status gxpo_slow_step(gxpo_ctx* c, void* stream) {
+    if (!c) return GXPO_ERR_INVALID_ARG;
+    if (c->phase != EXTRAPOLATED) return fail(c, GXPO_ERR_STATE, "slow step must follow extrapolate");
+    const TensorDesc none = {};
+    c->t_opt += 1;
+    StepParams p = make_step_params(c, 2, 0, 0, 0, 1);
+    gxpo_status st = launch_step(c, (cudaStream_t)stream, c->d_descs, c->d_chunks, c->num_chunks, none, p,
+                                 c->user_sumsq ? c->user_sumsq : c->d_sumsq);
+    if (st != GXPO_OK) { c->t_opt -= 1; return st; }
+    c->phase = SLOW_DONE;
+    return GXPO_OK;
+}
+
+gxpo_status gxpo_gate_update(gxpo_ctx* c, void* stream, gxpo_gate_result* out) {
+    if (!c) return GXPO_ERR_INVALID_ARG;
+    if (c->phase != SLOW_DONE) return fail(c, GXPO_ERR_STATE, "gate update must follow the slow step");
+    c->phase = IDLE;
+    return run_gate(c, (cudaStream_t)stream, c->user_sumsq ? c->user_sumsq : c->d_sumsq, out);
+}
+
+gxpo_status gxpo_set_sumsq_buffer(gxpo_ctx* c, double* sumsq_dev) {
+    if (!c) return GXPO_ERR_INVALID_ARG;
+    if (c->phase == SLOW_DONE) return fail(c, GXPO_ERR_STATE, "a norm is pending: call gxpo_gate_update first");
+    if (((uintptr_t)sumsq_dev) & 7u) return fail(c, GXPO_ERR_ALIGNMENT, "sumsq buffer must be 8-byte aligned");
+    c->user_sumsq = sumsq_dev;
+    return GXPO_OK;
+}
+
+gxpo_status gxpo_gate_peek(const gxpo_ctx* c, int* active, long long* s_star, long long* t) {
+    if (!c) return GXPO_ERR_INVALID_ARG;
+    if (active) *active = gate_active(c) ? 1 : 0;
+    if (s_star) *s_star = c->s_star;
+    if (t) *t = c->t;
+    return GXPO_OK;
+}
+
+long long gxpo_optimizer_steps(const gxpo_ctx* c) { return c ? c->t_opt : -1; }
+
+long long gxpo_backward_passes(const gxpo_ctx* c) {
+    if (!c) return -1;
+    const long long s = (c->s_star < 0 || c->s_star > c->t) ? c->t : c->s_star;
+    return 3 * s + (c->t - s);
+}
+
+long long gxpo_launch_count(const gxpo_ctx* c) { return c ? c->launches : -1; }
+
+const char* gxpo_last_error(const gxpo_ctx* c) { return c ? c->err : "null context"; }
+
+const char* gxpo_status_string(gxpo_status s) {
+    switch (s) {
+        case GXPO_OK: return "ok";
+        case GXPO_ERR_INVALID_ARG: return "invalid argument";
+        case GXPO_ERR_ALIGNMENT: return "misaligned pointer";
+        case GXPO_ERR_STATE: return "call out of order";
+        case GXPO_ERR_CUDA: return "CUDA error";
+        case GXPO_ERR_TIMEOUT: return "device-side wait timed out";
+        case GXPO_ERR_NONFINITE: return "non-finite gradient norm";
+    }
+    return "unknown status";
+}
+
+gxpo_status gxpo_tune(gxpo_ctx* c, int ctas_per_sm, int variant) {
+    if (!c) return GXPO_ERR_INVALID_ARG;
+    if (ctas_per_sm < 0 || ctas_per_sm > 16) return fail(c, GXPO_ERR_INVALID_ARG, "ctas_per_sm must be in [0, 16]");
+    if (variant < 0 || variant > 2) return fail(c, GXPO_ERR_INVALID_ARG, "variant must be 0, 1 or 2");
+    c->ctas_per_sm = ctas_per_sm;
+    c->variant = variant == 0 ? 2 : variant;
+    return GXPO_OK;
+}
+
+// ---- small-state checkpoint -------------------------------------------------
+namespace {
+struct StateHeader {
+    unsigned magic, version;
+    int window, head, count, pad;
+    long long t, s_star, t_opt;
+};
+constexpr unsigned kMagic = 0x4F505847u;   // "GXPO"
+}  // namespace
+
+gxpo_status gxpo_state_export(gxpo_ctx* c, void* buf, size_t* len) {
+    if (!c || !len) return GXPO_ERR_INVALID_ARG;
+    const size_t need = sizeof(StateHeader) + (size_t)c->cfg.window * sizeof(double);
+    if (!buf) { *len = need; return GXPO_OK; }
+    if (*len < need) { *len = need; return fail(c, GXPO_ERR_INVALID_ARG, "buffer too small: need %zu bytes", need); }
+    if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "state export in the middle of a step");
+    CUDA_TRY(c, cudaDeviceSynchronize());
+    GateState g;
+    CUDA_TRY(c, cudaMemcpy(&g, c->d_gate, sizeof(g), cudaMemcpyDeviceToHost));
+    StateHeader h;
+    std::memset(&h, 0, sizeof(h));
+    h.magic = kMagic; h.version = 1; h.window = c->cfg.window; h.head = g.head; h.count = g.count;
+    h.t = c->t; h.s_star = c->s_star; h.t_opt = c->t_opt;
+    std::memcpy(buf, &h, sizeof(h));
+    CUDA_TRY(c, cudaMemcpy(static_cast<char*>(buf) + sizeof(h), c->d_ring, (size_t)c->cfg.window * sizeof(double), cudaMemcpyDeviceToHost));
+    *len = need;
+    return GXPO_OK;
+}
+
+gxpo_status gxpo_state_import(gxpo_ctx* c, const void* buf, size_t len) {
+    if (!c || !buf) return GXPO_ERR_INVALID_ARG;
+    const size_t need = sizeof(StateHeader) + (size_t)c->cfg.window * sizeof(double);
+    if (len < need) return fail(c, GXPO_ERR_INVALID_ARG, "state blob too short");
+    if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "state import in the middle of a step");
+    StateHeader h;
+    std::memcpy(&h, buf, sizeof(h));
+    if (h.magic != kMagic || h.version != 1) return fail(c, GXPO_ERR_INVALID_ARG, "not a GXPO state blob");
+    if (h.window != c->cfg.window) return fail(c, GXPO_ERR_INVALID_ARG, "window mismatch: blob %d, context %d", h.window, c->cfg.window);
+    if (h.head < 0 || h.head >= h.window || h.count < 0 || h.count > h.window || h.t < 0 || h.t_opt < 0 || h.s_star < -1)
+        return fail(c, GXPO_ERR_INVALID_ARG, "corrupt state blob");
+    CUDA_TRY(c, cudaDeviceSynchronize());
+    GateState g;
+    g.head = h.head; g.count = h.count; g.s_star = h.s_star;
+    CUDA_TRY(c, cudaMemcpy(c->d_gate, &g, sizeof(g), cudaMemcpyHostToDevice));
+    CUDA_TRY(c, cudaMemcpy(c->d_ring, static_cast<const char*>(buf) + sizeof(h), (size_t)c->cfg.window * sizeof(double), cudaMemcpyHostToDevice));
+    c->t = h.t; c->s_star = h.s_star; c->t_opt = h.t_opt;
+    return GXPO_OK;
+}
+
+// ---- host-resident parameters ------------------------------------------------
+gxpo_status gxpo_step_host(gxpo_ctx* c, const gxpo_tensor* list, int count, long long staging_elems,
+                           void* stream, gxpo_gate_result* out) {
+    if (!c) return GXPO_ERR_INVALID_ARG;
+    if (count < 0 || (count > 0 && !list)) return fail(c, GXPO_ERR_INVALID_ARG, "bad list/count");
+    if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "host step in the middle of a device step");
+    if (staging_elems <= 0) staging_elems = 1LL << 24;
+    staging_elems = (staging_elems + kChunk - 1) / kChunk * kChunk;
+    for (int i = 0; i < count; ++i) {
+        gxpo_status s = check_tensor(c, list[i], i, false);
+        if (s != GXPO_OK) return s;
+    }
+    gxpo_status s0 = ensure_staging(c, staging_elems);
+    if (s0 != GXPO_OK) return s0;
+    Staging& st = c->stg;
+    cudaStream_t user = (cudaStream_t)stream;
+    const bool adamw = c->opt.kind == GXPO_OPT_ADAMW;
+    const bool active = gate_active(c);
+    const size_t gsz = (c->grad_dtype == GXPO_BF16) ? 2 : 4;
+    CUDA_TRY(c, cudaStreamSynchronize(user));
+    CUDA_TRY(c, cudaMemsetAsync(st.piece_sumsq, 0, 2 * sizeof(double), st.stream[0]));
+    CUDA_TRY(c, cudaStreamSynchronize(st.stream[0]));
+    const long long t_opt0 = c->t_opt;
+    int piece = 0;
+    for (int i = 0; i < count; ++i) {
+        const gxpo_tensor& T = list[i];
+        for (long long off = 0; off < T.n; off += staging_elems, ++piece) {
+            const long long len = (T.n - off < staging_elems) ? (T.n - off) : staging_elems;
+            const int k = piece & 1;
+            cudaStream_t s = st.stream[k];
+            // the slot is free once its previous piece has been copied back (same stream)
+            const size_t fb = (size_t)len * sizeof(float);
+            CUDA_TRY(c, cudaMemcpyAsync(st.theta[k], T.theta + off, fb, cudaMemcpyHostToDevice, s));
+            if (adamw) {
+                CUDA_TRY(c, cudaMemcpyAsync(st.m[k], T.m + off, fb, cudaMemcpyHostToDevice, s));
+                CUDA_TRY(c, cudaMemcpyAsync(st.v[k], T.v + off, fb, cudaMemcpyHostToDevice, s));
+            }
+            CUDA_TRY(c, cudaMemcpyAsync(st.g[k][0], static_cast<const char*>(T.g0) + off * gsz, len * gsz, cudaMemcpyHostToDevice, s));
+            if (active) {
+                CUDA_TRY(c, cudaMemcpyAsync(st.g[k][1], static_cast<const char*>(T.g1) + off * gsz, len * gsz, cudaMemcpyHostToDevice, s));
+                CUDA_TRY(c, cudaMemcpyAsync(st.g[k][2], static_cast<const char*>(T.g_slow) + off * gsz, len * gsz, cudaMemcpyHostToDevice, s));
+            }
+            TensorDesc d;
+            d.theta = st.theta[k]; d.work = st.work[k]; d.m = st.m[k]; d.v = st.v[k];
+            d.g[0] = st.g[k][0]; d.g[1] = st.g[k][1]; d.g[2] = st.g[k][2];
+            d.n = len;
+            const long long nch = (len + kChunk - 1) / kChunk;
+            gxpo_status rs;
+            if (active) {
+                // the kernels of a piece run back to back on the slot's stream; the
+                // norm's scratch is shared, which is safe because both slots' kernels
+                // are serialised through the `done` events below
+                if (piece > 0) CUDA_TRY(c, cudaStreamWaitEvent(s, st.done[k ^ 1], 0));
+                c->t_opt = t_opt0 + 1;
+                rs = launch_step(c, s, nullptr, nullptr, nch, d, make_step_params(c, 0, 0, 1, 0, 0), c->d_sumsq);
+                if (rs != GXPO_OK) return rs;
+                c->t_opt = t_opt0 + 2;
+                rs = launch_step(c, s, nullptr, nullptr, nch, d, make_step_params(c, 1, 1, 1, 0, 0), c->d_sumsq);
+                if (rs != GXPO_OK) return rs;
+                rs = launch_extrap(c, s, nullptr, nullptr, nch, d, make_extrap_params(c, GXPO_PLACE_PINGPONG));
+                if (rs != GXPO_OK) return rs;
+                c->t_opt = t_opt0 + 3;
+                rs = launch_step(c, s, nullptr, nullptr, nch, d, make_step_params(c, 2, 0, 0, 0, 1), st.piece_sumsq + 1);
+                if (rs != GXPO_OK) return rs;
+                accumulate_kernel<<<1, 32, 0, s>>>(st.piece_sumsq, st.piece_sumsq + 1);
+                c->launches += 1;
+                CUDA_TRY(c, cudaEventRecord(st.done[k], s));
+            } else {
+                c->t_opt = t_opt0 + 1;
+                rs = launch_step(c, s, nullptr, nullptr, nch, d, make_step_params(c, 0, 0, 0, 0, 0), c->d_sumsq);
+                if (rs != GXPO_OK) return rs;
+            }
+            CUDA_TRY(c, cudaMemcpyAsync(T.theta + off, st.theta[k], fb, cudaMemcpyDeviceToHost, s));
+            if (adamw) {
+                CUDA_TRY(c, cudaMemcpyAsync(T.m + off, st.m[k], fb, cudaMemcpyDeviceToHost, s));
+                CUDA_TRY(c, cudaMemcpyAsync(T.v + off, st.v[k], fb, cudaMemcpyDeviceToHost, s));
+            }
+        }
+    }
+    CUDA_TRY(c, cudaStreamSynchronize(st.stream[0]));
+    CUDA_TRY(c, cudaStreamSynchronize(st.stream[1]));
+    if (active) {
+        c->t_opt = t_opt0 + 3;
+        return run_gate(c, st.stream[0], st.piece_sumsq, out);
+    }
+    c->t_opt = t_opt0 + 1;
+    c->t += 1;
+    if (out) {
+        out->active = 0; out->tripped = 0; out->t = c->t; out->s_star = c->s_star;
+        out->norm = out->z = out->mu = out->sigma = std::nan("");
+    }
+    return GXPO_OK;
+}
+
+// ---- surrogate harness ---------------------------------------------------------
+gxpo_status gxpo_quad_grad(const float* theta, const float* a, const float* b, float* g, long long n, void* stream) {
+    if (n < 0 || (n > 0 && (!theta || !a || !b || !g))) return GXPO_ERR_INVALID_ARG;
+    if (n == 0) return GXPO_OK;
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    long long want = (n / 8 + kThreads - 1) / kThreads;
+    long long grid = (long long)sms * 8;
+    if (grid > want) grid = want < 1 ? 1 : want;
+    quad_grad_kernel<<<(int)grid, kThreads, 0, (cudaStream_t)stream>>>(theta, a, b, g, n);
+    return cudaGetLastError() == cudaSuccess ? GXPO_OK : GXPO_ERR_CUDA;
+}
+
+size_t gxpo_quad_scratch_bytes(void) { return kMaxGrid * sizeof(double) + 64; }
+
+gxpo_status gxpo_quad_active_step(float* theta, const float* a, const float* b, long long n, float lr, int K,
+                                  float alpha, float delta, float den_eps, double* sumsq_dev,
+                                  void* scratch_dev, void* stream) {
+    if (n < 0 || K < 2 || !sumsq_dev || !scratch_dev || (n > 0 && (!theta || !a || !b))) return GXPO_ERR_INVALID_ARG;
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    long long want = (n / 8 + kThreads - 1) / kThreads;
+    long long grid = (long long)sms * 8;
+    if (grid > want) grid = want < 1 ? 1 : want;
+    if (grid > kMaxGrid) grid = kMaxGrid;
+    QuadParams q;
+    q.lr = lr; q.alpha = alpha; q.delta = delta; q.den_eps = den_eps; q.K = K;
+    double* partials = static_cast<double*>(scratch_dev);
+    unsigned* ticket = reinterpret_cast<unsigned*>(static_cast<char*>(scratch_dev) + kMaxGrid * sizeof(double));
+    quad_active_kernel<<<(int)grid, kThreads, 0, (cudaStream_t)stream>>>(theta, a, b, n, q, partials, ticket, sumsq_dev);
+    return cudaGetLastError() == cudaSuccess ? GXPO_OK : GXPO_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,285 @@
+"""Parity of the CUDA library (through its C ABI) against the CPU oracle,
+element by element on the same seeded inputs.  Sizes span several 2048-element
+tiles, several 32768-element chunks and ragged tails."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import gxpo_oracle as ora
+from paper_2605_06755_b200 import workloads
+from tests import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+SIZES = [1, 7, 8, 2048, 2049, 40003, 3 * 32768 + 5]
+
+
+def _binding():
+    from paper_2605_06755_b200 import binding
+    return binding
+
+
+def _problem(n, seed, grad_dtype, warm=True, zero_frac=0.0, offset=0):
+    th, m, v, g0, g1, gs = workloads.llm_inputs_numpy(n, seed, grad_dtype, zero_frac, warm)
+    return gu.Problem(th, m, v, g0, g1, gs, offset_elems=offset)
+
+
+def _ctx(b, grad_dtype, **kw):
+    cfg, opt = b.make_cfg(**kw)
+    return b.Context(cfg, opt, b.BF16 if grad_dtype == "bf16" else b.F32), cfg, opt
+
+
+@pytest.mark.parametrize("n", SIZES)
+@pytest.mark.parametrize("grad_dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("kind", ["adamw", "gd"])
+@pytest.mark.parametrize("placement", [0, 1])
+def test_active_step_matches_oracle(n, grad_dtype, kind, placement):
+    b = _binding()
+    import torch
+    pr = _problem(n, seed=100 + n, grad_dtype=grad_dtype)
+    ctx, cfg, opt = _ctx(b, grad_dtype, kind=b.OPT_ADAMW if kind == "adamw" else b.OPT_GD,
+                         lr=1e-3, K=5, alpha=0.5, placement=placement)
+    gcfg, ocfg = gu.ora_cfgs(cfg, opt)
+    ctx.bind([pr.ptrs()])
+    st = pr.oracle_state(ocfg, t_opt=0)
+    grads = pr.oracle_grads()
+
+    # the oracle, step by step
+    theta0 = st.theta.copy()
+    st.optim_step(grads[0], True)
+    o_theta1, o_m1, o_v1 = st.theta.copy(), None if st.m is None else st.m.copy(), None if st.v is None else st.v.copy()
+    st.optim_step(grads[1], True)
+    o_theta2 = st.theta.copy()
+    o_tilde, _, o_scale = ora.extrapolate(theta0, o_theta2, grads[0], grads[1], gcfg.K, gcfg.alpha,
+                                          gcfg.delta, gcfg.den_eps, True, want_aux=True)
+    sat = ~np.isfinite(o_scale) | (np.abs(o_scale) > 1e30)
+    st.theta = o_tilde.copy()
+    st.optim_step(grads[2], True)
+    o_norm = ora.l2norm(grads[2])
+
+    # the library, call by call
+    ctx.probe_step(0)
+    live1 = pr.work if placement == 0 else pr.theta
+    gu.assert_close(gu.to_host_f64(live1), o_theta1, "theta1")
+    if placement == 1:
+        np.testing.assert_array_equal(gu.to_host_f64(pr.work), theta0)      # snapshot of theta^t
+    else:
+        np.testing.assert_array_equal(gu.to_host_f64(pr.theta), theta0)     # theta^t untouched
+    if kind == "adamw":
+        gu.assert_close(gu.to_host_f64(pr.m), o_m1, "m after probe 0")
+        gu.assert_close(gu.to_host_f64(pr.v), o_v1, "v after probe 0")
+    ctx.probe_step(1)
+    # theta2 starts from the library's own theta1 (within an ulp of the oracle's)
+    gu.assert_close(gu.to_host_f64(live1), o_theta2, "theta2", rtol=2e-6)
+    ctx.extrapolate()
+    # chained: (theta2 - theta0) cancels, the scale factor amplifies theta2's last-ulp
+    # differences; the strict per-call check is test_extrapolate_call_alone
+    slack = gu.displacement_slack(theta0, o_theta2, o_scale, gcfg.alpha)
+    gu.assert_close(gu.to_host_f64(pr.theta), o_tilde, "theta-tilde", saturated=sat, extra_abs=slack)
+    ctx.slow_step()
+    res = ctx.gate_update(allow_nonfinite=True)
+    torch.cuda.synchronize()
+    gu.assert_close(gu.to_host_f64(pr.theta), st.theta, "theta after slow step", saturated=sat,
+                    rtol=2e-6, extra_abs=slack)
+    if kind == "adamw":
+        gu.assert_close(gu.to_host_f64(pr.m), st.m, "m after slow step")
+        gu.assert_close(gu.to_host_f64(pr.v), st.v, "v after slow step")
+    assert res.norm == pytest.approx(o_norm, rel=gu.RTOL_NORM)
+    assert ctx.optimizer_steps() == 3 and res.t == 1 and res.active == 1
+    assert math.isnan(res.z)
+    ctx.close()
+
+
+def _run_extrapolate_alone(b, theta0, theta2, g0d, g1d, grad_dtype, kind, placement, **kw):
+    """gxpo_extrapolate on given theta^t and theta^{t,2}: the library's own probe
+    steps with lr = 0 are identities and put the context in the right state; the
+    two points are then written where the placement expects them."""
+    n = theta0.size
+    dummy = np.zeros(n, dtype=np.float32)
+    pr = gu.Problem(theta0, dummy if kind == "adamw" else None, dummy if kind == "adamw" else None,
+                    g0d, g1d, g0d)
+    ctx, cfg, opt = _ctx(b, grad_dtype, kind=b.OPT_ADAMW if kind == "adamw" else b.OPT_GD, lr=0.0,
+                         weight_decay=0.0, placement=placement, **kw)
+    ctx.bind([pr.ptrs()])
+    ctx.probe_step(0)
+    ctx.probe_step(1)
+    if placement == 0:
+        pr.theta.copy_(gu.to_dev(theta0)); pr.work.copy_(gu.to_dev(theta2))
+    else:
+        pr.theta.copy_(gu.to_dev(theta2)); pr.work.copy_(gu.to_dev(theta0))
+    ctx.extrapolate()
+    got = gu.to_host_f64(pr.theta)
+    ctx.close()
+    return got
+
+
+@pytest.mark.parametrize("K", [3, 5, 10])
+@pytest.mark.parametrize("grad_dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("placement", [0, 1])
+def test_extrapolate_call_alone(K, grad_dtype, placement):
+    """Strict 1e-6 check of the extrapolation call on seeded theta^t, theta^{t,2}, g0, g1
+    with the heavy-tailed ratios of the LLM-shaped recipe, 3 % inactive coordinates."""
+    b = _binding()
+    n = 2 * 32768 + 1234
+    th, _, _, g0, g1, _ = workloads.llm_inputs_numpy(n, seed=900 + K, grad_dtype=grad_dtype, zero_frac=0.03)
+    rng = np.random.default_rng(K)
+    theta2 = (th + 2e-3 * rng.standard_normal(n)).astype(np.float32)
+    got = _run_extrapolate_alone(b, th, theta2, g0, g1, grad_dtype, "adamw", placement, K=K, alpha=0.5)
+    want, _, scale = ora.extrapolate(th.astype(np.float64), theta2.astype(np.float64), gu.grad_to_f64(g0),
+                                     gu.grad_to_f64(g1), K, 0.5, 1e-8, 0.0, True, want_aux=True)
+    sat = ~np.isfinite(scale) | (np.abs(scale) > 1e30)
+    gu.assert_close(got, want, f"theta-tilde K={K}", saturated=sat)
+    assert 0.02 < (scale == 1.0).mean() < 0.05
+
+
+@pytest.mark.parametrize("K", [2, 3, 4, 5, 10])
+@pytest.mark.parametrize("grad_dtype", ["bf16", "f32"])
+def test_extrapolate_edge_values(K, grad_dtype):
+    """r = +-1, |g0| = delta exactly, zeros, huge and tiny ratios, negative ratios."""
+    b = _binding()
+    delta = np.float32(2.0 ** -20)                      # exact in bfloat16 too
+    g0 = np.array([1.0, 1.0, delta, -delta, 0.0, 2.0 ** -19, 1.0, -1.0, 2.0 ** -19, 0.5, 3.0, -0.25,
+                   1.0, 1.0, 2.0, 1.0], dtype=np.float32)
+    g1 = np.array([1.0, -1.0, 5.0, 5.0, 1.0, 2.0 ** 10, 0.0, -0.999, -2.0 ** 12, 0.4375, -3.0, 0.75,
+                   -0.9921875, -1.0078125, -1.0, 1.5], dtype=np.float32)
+    rng = np.random.default_rng(K)
+    reps = 700                                          # 11200 elements: several tiles
+    g0 = np.tile(g0, reps)
+    g1 = np.tile(g1, reps)
+    n = g0.size
+    theta0 = rng.standard_normal(n).astype(np.float32)
+    theta2 = (theta0 + 1e-2 * rng.standard_normal(n)).astype(np.float32)
+    if grad_dtype == "bf16":
+        g0d, g1d = workloads.f32_to_bf16_bits(g0), workloads.f32_to_bf16_bits(g1)
+        np.testing.assert_array_equal(workloads.bf16_bits_to_f32(g0d), g0)   # all exact in bf16
+        np.testing.assert_array_equal(workloads.bf16_bits_to_f32(g1d), g1)
+    else:
+        g0d, g1d = g0, g1
+    for den_eps in (0.0, 2.0 ** -6):
+        # place theta^t in `theta` and theta^{t,2} in `work` (PINGPONG layout) by hand:
+        # run the library's own probe steps with lr = 0 so that they are identities
+        pr = gu.Problem(theta0, None, None, g0d, g1d, g0d)
+        ctx, cfg, opt = _ctx(b, grad_dtype, kind=b.OPT_GD, lr=0.0, K=K, alpha=0.5, delta=float(delta),
+                             den_eps=den_eps)
+        ctx.bind([pr.ptrs()])
+        ctx.probe_step(0)
+        ctx.probe_step(1)
+        pr.work.copy_(gu.to_dev(theta2))
+        ctx.extrapolate()
+        want, _, scale = ora.extrapolate(theta0.astype(np.float64), theta2.astype(np.float64),
+                                         g0.astype(np.float64), g1.astype(np.float64), K, 0.5,
+                                         float(delta), den_eps, True, want_aux=True)
+        sat = ~np.isfinite(scale) | (np.abs(scale) > 1e30)
+        got = gu.to_host_f64(pr.theta)
+        gu.assert_close(got, want, f"K={K} den_eps={den_eps}", saturated=sat)
+        # r = -1 with the literal formula: both sides non-finite
+        if den_eps == 0.0:
+            assert not np.isfinite(want[1]) and not np.isfinite(got[1])
+            assert np.all(np.isfinite(got[2:5]))       # |g0| <= delta: scale 1, finite
+        else:
+            assert np.isfinite(got[1]) and np.isfinite(got[12])   # guarded: scale 1
+        ctx.close()
+
+
+def test_multi_tensor_list_with_odd_sizes_and_misaligned_tensors():
+    b = _binding()
+    sizes = [512, 3584, 1, 70001, 2 * 32768, 33, 32768 + 2047, 5]
+    offsets = [0, 0, 0, 1, 0, 3, 2, 0]                  # element offsets -> misaligned pointers
+    probs = [_problem(n, seed=7 + i, grad_dtype="bf16", zero_frac=0.03, offset=off)
+             for i, (n, off) in enumerate(zip(sizes, offsets))]
+    ctx, cfg, opt = _ctx(b, "bf16", lr=1e-3, K=10, alpha=0.5)
+    gcfg, ocfg = gu.ora_cfgs(cfg, opt)
+    ctx.bind([p.ptrs() for p in probs])
+    res = ctx.active_step(allow_nonfinite=True)
+    sumsq = 0.0
+    for i, p in enumerate(probs):
+        st = p.oracle_state(ocfg)
+        grads = p.oracle_grads()
+        trace = {}
+        ora.active_step(st, gcfg, lambda w, th: grads[w], round_f32=True, trace=trace)
+        sat = ~np.isfinite(trace["scale"]) | (np.abs(trace["scale"]) > 1e30)
+        slack = gu.displacement_slack(p.np_in["theta"].astype(np.float64), trace["theta2"],
+                                      trace["scale"], gcfg.alpha)
+        gu.assert_close(gu.to_host_f64(p.theta), st.theta, f"tensor {i} theta", saturated=sat,
+                        rtol=2e-6, extra_abs=slack)
+        gu.assert_close(gu.to_host_f64(p.m), st.m, f"tensor {i} m")
+        gu.assert_close(gu.to_host_f64(p.v), st.v, f"tensor {i} v")
+        sumsq += ora.sum_squares(grads[2])
+        if p.n >= 3584:
+            assert (trace["scale"] == 1.0).mean() > 0.01    # the inactive branch was exercised
+    assert res.norm == pytest.approx(math.sqrt(sumsq), rel=gu.RTOL_NORM)
+    ctx.close()
+
+
+def test_empty_list_and_empty_tensor():
+    b = _binding()
+    ctx, cfg, opt = _ctx(b, "bf16")
+    ctx.bind([])
+    res = ctx.active_step()
+    assert res.norm == 0.0 and res.t == 1
+    pr = _problem(100, 1, "bf16")
+    empty = b.TensorPtrs(0, 0, 0, 0, 0, 0, 0, 0)
+    before = gu.to_host_f64(pr.theta)
+    ctx.bind([empty, pr.ptrs(), empty])
+    res = ctx.active_step()
+    assert res.norm == pytest.approx(ora.l2norm(pr.oracle_grads()[2]), rel=gu.RTOL_NORM)
+    assert not np.array_equal(gu.to_host_f64(pr.theta), before)
+    ctx.close()
+
+
+def test_access_variants_and_launch_shapes_agree_bitwise():
+    b = _binding()
+    n = 5 * 32768 + 77
+    outs = []
+    for variant, ctas in [(1, 0), (2, 0), (2, 1), (1, 7)]:
+        pr = _problem(n, seed=42, grad_dtype="bf16")
+        ctx, cfg, opt = _ctx(b, "bf16", lr=1e-3, K=5)
+        ctx.tune(ctas, variant)
+        ctx.bind([pr.ptrs()])
+        res = ctx.active_step(allow_nonfinite=True)
+        outs.append((gu.to_host_f64(pr.theta), gu.to_host_f64(pr.m), gu.to_host_f64(pr.v), res.norm))
+        ctx.close()
+    for o in outs[1:]:
+        for a, c in zip(o[:3], outs[0][:3]):
+            np.testing.assert_array_equal(a, c)
+        assert o[3] == pytest.approx(outs[0][3], rel=1e-12)
+
+
+def test_run_to_run_determinism():
+    b = _binding()
+    n = 3 * 32768 + 11
+    got = []
+    for _ in range(2):
+        pr = _problem(n, seed=5, grad_dtype="bf16")
+        ctx, cfg, opt = _ctx(b, "bf16", lr=1e-3)
+        ctx.bind([pr.ptrs()])
+        res = ctx.active_step(allow_nonfinite=True)
+        got.append((gu.to_host_f64(pr.theta), res.norm))
+        ctx.close()
+    np.testing.assert_array_equal(got[0][0], got[1][0])
+    assert got[0][1] == got[1][1]                       # bitwise: fixed summation order
+
+
+def test_probe_step_against_library_adamw_on_device():
+    """The fallback step is one AdamW step: cross-check with torch.optim.AdamW (fp32)."""
+    b = _binding()
+    import torch
+    n = 100003
+    pr = _problem(n, seed=9, grad_dtype="f32", warm=False)
+    ctx, cfg, opt = _ctx(b, "f32", lr=1e-3)
+    ctx.bind([pr.ptrs()])
+    p = torch.nn.Parameter(pr.theta.clone())
+    lib = torch.optim.AdamW([p], lr=1e-3, betas=(0.9, 0.999), eps=1e-8, weight_decay=0.01)
+    for g in (pr.g0, pr.g1):
+        p.grad = g.clone()
+        lib.step()
+        pr.g0.copy_(g)
+        ctx.probe_step(-1)
+    torch.cuda.synchronize()
+    got, want = pr.theta.double().cpu().numpy(), p.detach().double().cpu().numpy()
+    gu.assert_close(got, want, "theta vs torch AdamW", rtol=2e-6)
+    gu.assert_close(pr.m.double().cpu().numpy(), lib.state[p]["exp_avg"].double().cpu().numpy(), "m", rtol=2e-6)
+    gu.assert_close(pr.v.double().cpu().numpy(), lib.state[p]["exp_avg_sq"].double().cpu().numpy(), "v", rtol=2e-6)
+    assert ctx.gate_peek()[2] == 2 and ctx.optimizer_steps() == 2
+    ctx.close()
