@@ -30,7 +30,7 @@ METRIC = "GXPO active-step params/sec"
 UNIT = "params/s"
 BYTES_STEP_ADAMW = 26      # R theta, m, v (12) + g bf16 (2); W theta, m, v (12)
 BYTES_EXTRAP = 16          # R theta2, theta0 (8) + g0, g1 bf16 (4); W theta-tilde (4)
-BYTES_ACTIVE = {0: 94, 1: 98}   # per placement: PINGPONG, SNAPSHOT (+4: theta^t copy)
+BYTES_FUSED = 32           # R theta1, theta0, m, v (16) + g0, g1 (4); W theta-tilde, m, v (12)
 
 
 def parse_args():
@@ -40,7 +40,8 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="qwen25_7b",
-                    choices=["qwen25_7b", "llama31_8b", "flat_1p54b", "small"])
+                    choices=["qwen25_7b", "llama31_8b", "flat_1p54b", "small", "flat"])
+    ap.add_argument("--params", type=int, default=1 << 26, help="size of the 'flat' workload")
     ap.add_argument("--layers", type=int, default=0, help="override the decoder depth (0 = full)")
     ap.add_argument("--K", type=int, default=5)
     ap.add_argument("--alpha", type=float, default=0.5)
@@ -48,7 +49,10 @@ def parse_args():
     ap.add_argument("--placement", type=int, default=0)
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--ctas", type=int, default=0)
+    ap.add_argument("--unit-tiles", type=int, default=0)
     ap.add_argument("--fallback", action="store_true", help="time the single-pass fallback step")
+    ap.add_argument("--unfused", action="store_true",
+                    help="probe step 1 and extrapolate as two sweeps (94 B/param) instead of one (84)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-params", type=int, default=1 << 26)
@@ -62,6 +66,8 @@ def workload_shapes(args):
         return w.qwen25_7b_shapes(args.layers or 28), "Qwen2.5-7B-shaped tensor list"
     if args.workload == "llama31_8b":
         return w.llama31_8b_shapes(args.layers or 32), "Llama-3.1-8B-shaped tensor list"
+    if args.workload == "flat":
+        return [("flat", args.params)], f"flat {args.params}-parameter buffer"
     if args.workload == "flat_1p54b":
         return [("flat", w.FLAT_QWEN25_1P5B)], "flat 1.54e9-parameter buffer"
     return w.qwen25_7b_shapes(args.layers or 1), "Qwen2.5-7B-shaped list, reduced depth"
@@ -148,9 +154,7 @@ def oracle_sample(n, seed, K, alpha, lr):
     from paper_2605_06755_b200 import workloads as w
     th, m, v, g0, g1, gs = w.llm_inputs_numpy(n, seed, "bf16")
     grads = [ora.bf16_bits_to_f64(g) for g in (g0, g1, gs)]
-    opt = ora.OptCfg(kind="adamw", lr=float(np.float32(lr)), beta1=float(np.float32(0.9)),
-                     beta2=float(np.float32(0.999)), eps=float(np.float32(1e-8)),
-                     weight_decay=float(np.float32(0.01)))
+    opt = ora.OptCfg(kind="adamw", lr=lr, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
     cfg = ora.GxpoCfg(K=K, alpha=alpha, delta=float(np.float32(1e-8)))
     st = ora.State(th, opt, m, v)
     return ora, st, cfg, grads
@@ -257,27 +261,39 @@ def run_ours(args):
 
     cfg, opt = b.make_cfg(K=args.K, alpha=args.alpha, lr=args.lr, placement=args.placement)
     ctx = b.Context(cfg, opt, b.BF16)
-    ctx.tune(args.ctas, args.variant)
+    ctx.tune(args.ctas, args.variant, args.unit_tiles)
     ctx.bind(ptrs)
     if world > 1:
         ctx.set_sumsq_buffer(sumsq.data_ptr())
 
-    n_ev = 5
+    fused = not args.unfused
+    names = ["probe_step0", "probe_extrapolate", "slow_step"] if fused else \
+        ["probe_step0", "probe_step1", "extrapolate", "slow_step"]
+    if args.fallback:
+        names = ["fallback_step"]
+    n_ev = len(names) + 1
+
     def one_step(evs=None):
+        def mark(i):
+            if evs:
+                evs[i].record(stream)
+        mark(0)
         if args.fallback:
-            if evs: evs[0].record(stream)
             ctx.probe_step(-1, stream)
-            if evs: evs[1].record(stream)
+            mark(1)
             return None
-        if evs: evs[0].record(stream)
         ctx.probe_step(0, stream)
-        if evs: evs[1].record(stream)
-        ctx.probe_step(1, stream)
-        if evs: evs[2].record(stream)
-        ctx.extrapolate(stream)
-        if evs: evs[3].record(stream)
+        mark(1)
+        if fused:
+            ctx.probe_extrapolate(stream)
+            mark(2)
+        else:
+            ctx.probe_step(1, stream)
+            mark(2)
+            ctx.extrapolate(stream)
+            mark(3)
         ctx.slow_step(stream)
-        if evs: evs[4].record(stream)
+        mark(n_ev - 1)
         if world > 1:
             dist.all_reduce(sumsq)        # the one exchange of a sharded step: 8 bytes
         return ctx.gate_update(stream, allow_nonfinite=True)
@@ -315,29 +331,27 @@ def run_ours(args):
     ms_step = ms_total / args.steps
 
     # per-kernel durations from the events inside the timed region
-    names = ["probe_step0", "probe_step1", "extrapolate", "slow_step"]
-    per = {}
-    if not args.fallback:
-        for i, nm in enumerate(names):
-            per[nm] = statistics.mean(evs[s][i].elapsed_time(evs[s][i + 1]) for s in range(args.steps))
-        step_ms = statistics.mean([per["probe_step0"], per["probe_step1"], per["slow_step"]])
-    else:
-        per["fallback_step"] = statistics.mean(evs[s][0].elapsed_time(evs[s][1]) for s in range(args.steps))
-        step_ms = per["fallback_step"]
-
+    per = {nm: statistics.mean(evs[s][i].elapsed_time(evs[s][i + 1]) for s in range(args.steps))
+           for i, nm in enumerate(names)}
     peak, peak_kind = measured_peak_gbs()
-    bytes_probe0 = BYTES_STEP_ADAMW + (4 if args.placement == 1 else 0)
-    alg_bytes = {"probe_step0": bytes_probe0, "probe_step1": BYTES_STEP_ADAMW, "extrapolate": BYTES_EXTRAP,
-                 "slow_step": BYTES_STEP_ADAMW, "fallback_step": BYTES_STEP_ADAMW}
-    kernels = {nm: {"ms": ms, "gbs": alg_bytes[nm] * d / (ms * 1e-3) / 1e9} for nm, ms in per.items()}
-    achieved = BYTES_STEP_ADAMW * d / (step_ms * 1e-3) / 1e9 if args.placement == 0 or args.fallback else \
-        statistics.mean([kernels["probe_step1"]["gbs"], kernels["slow_step"]["gbs"]])
+    alg_bytes = {"probe_step0": BYTES_STEP_ADAMW + (4 if args.placement == 1 else 0),
+                 "probe_step1": BYTES_STEP_ADAMW, "extrapolate": BYTES_EXTRAP,
+                 "probe_extrapolate": BYTES_FUSED, "slow_step": BYTES_STEP_ADAMW,
+                 "fallback_step": BYTES_STEP_ADAMW}
+    kernels = {nm: {"ms": ms, "bytes_per_param": alg_bytes[nm],
+                    "gbs": alg_bytes[nm] * d / (ms * 1e-3) / 1e9} for nm, ms in per.items()}
+    # dominant kernel: the AdamW sweep (step_kernel), launched for probe step 0 (PINGPONG
+    # placement: plain 26 B/param), the slow step and the fallback step
+    dom = [nm for nm in ("probe_step0", "probe_step1", "slow_step", "fallback_step")
+           if nm in per and alg_bytes[nm] == BYTES_STEP_ADAMW]
+    step_ms = statistics.mean(per[nm] for nm in dom)
+    achieved = BYTES_STEP_ADAMW * d / (step_ms * 1e-3) / 1e9
     tpp = recorded_traffic_per_param()
-    roofline = {"bound": "hbm", "kernel": "step_kernel (AdamW sweep: probe steps, slow step, fallback)",
+    roofline = {"bound": "hbm", "kernel": "step_kernel (AdamW sweep: probe step, slow step, fallback step)",
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_kind": f"of {peak_kind}", "traffic": (tpp * d if tpp else None),
-                "algorithmic_bytes_per_launch": BYTES_STEP_ADAMW * d}
-    step_bytes = (BYTES_STEP_ADAMW if args.fallback else BYTES_ACTIVE[args.placement]) * d
+                "algorithmic_bytes_per_launch": BYTES_STEP_ADAMW * d, "launches_averaged": dom}
+    step_bytes = sum(alg_bytes[nm] for nm in names) * d
     whole_gbs = step_bytes / (ms_step * 1e-3) / 1e9
 
     total_params = d * world
@@ -348,7 +362,9 @@ def run_ours(args):
         "config": {"workload": desc, "params_per_gpu": d, "tensors": len(shapes), "optimizer": "AdamW",
                    "K": args.K, "alpha": args.alpha, "lr": args.lr, "grad_dtype": "bf16",
                    "placement": ["pingpong", "snapshot"][args.placement],
-                   "step": "fallback (single pass)" if args.fallback else "active (probe, probe, extrapolate, slow step, gate)",
+                   "step": "fallback (single pass)" if args.fallback else
+                   ("active (probe, fused probe+extrapolate, slow step, gate)" if fused else
+                    "active (probe, probe, extrapolate, slow step, gate)"),
                    "g_slow_aliases_g0": alias, "l2": "inputs larger than L2 (no flush needed)",
                    "parallelism": f"dp{world} (independent shards, one 8-byte all-reduce per step)" if world > 1 else "1 GPU"},
         "hbm_gbs_whole_step": whole_gbs, "hbm_frac_whole_step": whole_gbs / peak,
@@ -384,7 +400,7 @@ def run_e2e(torch, b, args, cfg, opt):
     pin = [torch.from_numpy(x.view(np.int16) if x.dtype == np.uint16 else x).pin_memory()
            for x in (th, m, v, g0, g1, gs)]
     ctx = b.Context(cfg, opt, b.BF16)
-    ctx.tune(args.ctas, args.variant)
+    ctx.tune(args.ctas, args.variant, args.unit_tiles)
     t = [b.tensor_ptrs(pin[0], None, pin[1], pin[2], pin[3], pin[4], pin[5])]
     l0 = None
     for i in range(2 + 3):

@@ -70,7 +70,11 @@ enum { GXPO_PLACE_PINGPONG = 0, GXPO_PLACE_SNAPSHOT = 1 };
  * The step count t advances on EVERY optimizer step, probes included (Sec. 2.3). */
 typedef struct {
     int kind; /* GXPO_OPT_GD or GXPO_OPT_ADAMW */
-    float lr, beta1, beta2, eps, weight_decay;
+    /* Doubles, as trainers hold them: the float32 constants the kernels use (beta,
+     * 1-beta, 1-lr*wd, lr/(1-beta1^t), 1/sqrt(1-beta2^t)) are each formed in double
+     * and rounded once, so beta2 = 0.999 gives 1-beta2 = float(0.001), not
+     * 1 - float(0.999). */
+    double lr, beta1, beta2, eps, weight_decay;
 } gxpo_opt_cfg;
 
 /* Hyper-parameters of Algorithm 1 ("Require" line) and of the adaptive rule.
@@ -152,6 +156,12 @@ gxpo_status gxpo_probe_step(gxpo_ctx* ctx, int which, void* stream);
  * state: PROBED1 -> EXTRAPOLATED. */
 gxpo_status gxpo_extrapolate(gxpo_ctx* ctx, void* stream);
 
+/* gxpo_probe_step(ctx, 1) and gxpo_extrapolate in ONE sweep: Algorithm 1 takes no
+ * backward pass at theta^{t,2}, so that point never has to reach memory.  Same
+ * per-coordinate arithmetic, bit-identical theta-tilde, m and v; 32 instead of
+ * 26 + 16 bytes per parameter.  state: PROBED0 -> EXTRAPOLATED. */
+gxpo_status gxpo_probe_extrapolate(gxpo_ctx* ctx, void* stream);
+
 /* Algorithm 1, "slow correction": theta^{t+1} <- OptimStep(theta-tilde, g_slow), in
  * place in `theta`, and sum(g_slow^2) accumulated in the same sweep (float64,
  * deterministic for a fixed launch shape).  state: EXTRAPOLATED -> SLOW_DONE. */
@@ -202,11 +212,12 @@ gxpo_status gxpo_state_import(gxpo_ctx* ctx, const void* buf, size_t len);
 gxpo_status gxpo_step_host(gxpo_ctx* ctx, const gxpo_tensor* list, int count,
                            long long staging_elems, void* stream, gxpo_gate_result* out);
 
-/* Launch-shape knobs, for benchmarking: resident CTAs per SM (0 = default) and the
- * memory-access variant (0 = default, 1 = 128-bit loads, 2 = 256-bit loads,
- * 3 = bulk-copy shared-memory ring).  Results are identical across variants except
- * for the summation order of the norm. */
-gxpo_status gxpo_tune(gxpo_ctx* ctx, int ctas_per_sm, int variant);
+/* Launch-shape knobs, for benchmarking: resident CTAs per SM (0 = default), the
+ * memory-access variant (0 = default, 1 = 128-bit loads, 2 = 256-bit loads) and the
+ * number of 2048-element tiles a CTA takes per round-robin turn (0 = default; 1, 2,
+ * 4, 8 or 16).  Element-wise results are identical across all settings; only the
+ * summation order of the norm changes. */
+gxpo_status gxpo_tune(gxpo_ctx* ctx, int ctas_per_sm, int variant, int unit_tiles);
 
 /* Number of kernels this context has launched so far. */
 long long gxpo_launch_count(const gxpo_ctx* ctx);

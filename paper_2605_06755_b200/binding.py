@@ -29,9 +29,9 @@ PLACE_PINGPONG, PLACE_SNAPSHOT = 0, 1
 
 
 class OptCfg(ctypes.Structure):
-    _fields_ = [("kind", ctypes.c_int), ("lr", ctypes.c_float), ("beta1", ctypes.c_float),
-                ("beta2", ctypes.c_float), ("eps", ctypes.c_float),
-                ("weight_decay", ctypes.c_float)]
+    _fields_ = [("kind", ctypes.c_int), ("lr", ctypes.c_double), ("beta1", ctypes.c_double),
+                ("beta2", ctypes.c_double), ("eps", ctypes.c_double),
+                ("weight_decay", ctypes.c_double)]
 
 
 class Cfg(ctypes.Structure):
@@ -63,6 +63,7 @@ _sigs = {
     "gxpo_bind": (ctypes.c_int, [_vp, ctypes.POINTER(Tensor), ctypes.c_int]),
     "gxpo_probe_step": (ctypes.c_int, [_vp, ctypes.c_int, _vp]),
     "gxpo_extrapolate": (ctypes.c_int, [_vp, _vp]),
+    "gxpo_probe_extrapolate": (ctypes.c_int, [_vp, _vp]),
     "gxpo_slow_step": (ctypes.c_int, [_vp, _vp]),
     "gxpo_gate_update": (ctypes.c_int, [_vp, _vp, ctypes.POINTER(GateResult)]),
     "gxpo_set_sumsq_buffer": (ctypes.c_int, [_vp, _vp]),
@@ -75,7 +76,7 @@ _sigs = {
     "gxpo_state_import": (ctypes.c_int, [_vp, _vp, ctypes.c_size_t]),
     "gxpo_step_host": (ctypes.c_int, [_vp, ctypes.POINTER(Tensor), ctypes.c_int,
                                       ctypes.c_longlong, _vp, ctypes.POINTER(GateResult)]),
-    "gxpo_tune": (ctypes.c_int, [_vp, ctypes.c_int, ctypes.c_int]),
+    "gxpo_tune": (ctypes.c_int, [_vp, ctypes.c_int, ctypes.c_int, ctypes.c_int]),
     "gxpo_launch_count": (ctypes.c_longlong, [_vp]),
     "gxpo_last_error": (ctypes.c_char_p, [_vp]),
     "gxpo_status_string": (ctypes.c_char_p, [ctypes.c_int]),
@@ -186,6 +187,9 @@ class Context:
     def extrapolate(self, stream=None):
         self._check(_lib.gxpo_extrapolate(self._h, _stream_ptr(stream)))
 
+    def probe_extrapolate(self, stream=None):
+        self._check(_lib.gxpo_probe_extrapolate(self._h, _stream_ptr(stream)))
+
     def slow_step(self, stream=None):
         self._check(_lib.gxpo_slow_step(self._h, _stream_ptr(stream)))
 
@@ -232,18 +236,21 @@ class Context:
         self._check(st)
         return res
 
-    def tune(self, ctas_per_sm: int = 0, variant: int = 0):
-        self._check(_lib.gxpo_tune(self._h, ctas_per_sm, variant))
+    def tune(self, ctas_per_sm: int = 0, variant: int = 0, unit_tiles: int = 0):
+        self._check(_lib.gxpo_tune(self._h, ctas_per_sm, variant, unit_tiles))
 
     def launch_count(self) -> int:
         return _lib.gxpo_launch_count(self._h)
 
     # -- convenience: the calls of one active step in Algorithm 1's order, for callers
     #    whose three gradient buffers are already filled (benchmarks, replay) --------
-    def active_step(self, stream=None, allow_nonfinite: bool = False) -> GateResult:
+    def active_step(self, stream=None, allow_nonfinite: bool = False, fused: bool = False) -> GateResult:
         self.probe_step(0, stream)
-        self.probe_step(1, stream)
-        self.extrapolate(stream)
+        if fused:
+            self.probe_extrapolate(stream)
+        else:
+            self.probe_step(1, stream)
+            self.extrapolate(stream)
         self.slow_step(stream)
         return self.gate_update(stream, allow_nonfinite)
 

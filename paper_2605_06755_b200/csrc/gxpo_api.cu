@@ -14,6 +14,11 @@ using namespace gxpo;
 
 namespace {
 
+constexpr int kDefaultUnitShift = 0;   // whole chunks
+constexpr int kDefaultCtasStep = 2;    // measured best for the 14R/12W sweep
+constexpr int kDefaultCtasExtrap = 4;  // the extrapolation needs more warps to cover its arithmetic
+constexpr int kDefaultCtasFused = 3;
+
 enum Phase { IDLE = 0, PROBED0 = 1, PROBED1 = 2, EXTRAPOLATED = 3, SLOW_DONE = 4 };
 
 struct Staging {                       // device pieces for gxpo_step_host
@@ -39,6 +44,7 @@ struct gxpo_ctx {
     int sm_count;
     int ctas_per_sm;                   // 0 = default
     int variant;                       // 1 = 128-bit, 2 = 256-bit
+    int unit_shift;                    // work unit = kChunk >> unit_shift elements
     Phase phase;
     // bound list
     TensorDesc* d_descs;
@@ -59,6 +65,9 @@ struct gxpo_ctx {
     // host mirror
     long long t, s_star, t_opt;
     long long launches;
+    const void* occ_key[32];           // resident CTAs per SM, per kernel (cache)
+    int occ_val[32];
+    int occ_n;
     Staging stg;
     char err[512];
 };
@@ -97,22 +106,34 @@ gxpo_status check_cfg(gxpo_ctx* c, const gxpo_cfg* g, const gxpo_opt_cfg* o, int
     if (g->placement != GXPO_PLACE_PINGPONG && g->placement != GXPO_PLACE_SNAPSHOT)
         return fail(c, GXPO_ERR_INVALID_ARG, "unknown placement %d", g->placement);
     if (o->kind != GXPO_OPT_GD && o->kind != GXPO_OPT_ADAMW) return fail(c, GXPO_ERR_INVALID_ARG, "unknown optimizer kind %d", o->kind);
-    if (!finite_f(o->lr)) return fail(c, GXPO_ERR_INVALID_ARG, "lr is not finite");
+    if (!std::isfinite(o->lr)) return fail(c, GXPO_ERR_INVALID_ARG, "lr is not finite");
     if (o->kind == GXPO_OPT_ADAMW) {
-        if (!(o->beta1 >= 0.0f && o->beta1 < 1.0f) || !(o->beta2 >= 0.0f && o->beta2 < 1.0f))
+        if (!(o->beta1 >= 0.0 && o->beta1 < 1.0) || !(o->beta2 >= 0.0 && o->beta2 < 1.0))
             return fail(c, GXPO_ERR_INVALID_ARG, "betas must be in [0, 1)");
-        if (!(o->eps >= 0.0f) || !finite_f(o->eps)) return fail(c, GXPO_ERR_INVALID_ARG, "eps must be finite and >= 0");
-        if (!finite_f(o->weight_decay)) return fail(c, GXPO_ERR_INVALID_ARG, "weight_decay is not finite");
+        if (!(o->eps >= 0.0) || !std::isfinite(o->eps)) return fail(c, GXPO_ERR_INVALID_ARG, "eps must be finite and >= 0");
+        if (!std::isfinite(o->weight_decay)) return fail(c, GXPO_ERR_INVALID_ARG, "weight_decay is not finite");
     }
     if (grad_dtype != GXPO_F32 && grad_dtype != GXPO_BF16) return fail(c, GXPO_ERR_INVALID_ARG, "unknown gradient dtype %d", grad_dtype);
     return GXPO_OK;
 }
 
-int grid_for(const gxpo_ctx* c, long long num_chunks, int default_per_sm) {
-    const int per_sm = c->ctas_per_sm > 0 ? c->ctas_per_sm : default_per_sm;
+// Persistent grid: CTAs per SM (tuned or default) clamped to what is actually resident
+// for this kernel, times the SM count.  Work is dealt round-robin, so a grid that is
+// only partly resident would leave a tail wave running alone.
+int grid_for(gxpo_ctx* c, const void* kernel, long long units, int default_per_sm) {
+    int per_sm = c->ctas_per_sm > 0 ? c->ctas_per_sm : default_per_sm;
+    int resident = 0;
+    for (int i = 0; i < c->occ_n; ++i)
+        if (c->occ_key[i] == kernel) resident = c->occ_val[i];
+    if (resident == 0) {
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kernel, kThreads, 0) != cudaSuccess || resident < 1)
+            resident = 1;
+        if (c->occ_n < 32) { c->occ_key[c->occ_n] = kernel; c->occ_val[c->occ_n] = resident; c->occ_n += 1; }
+    }
+    if (per_sm > resident) per_sm = resident;
     long long g = (long long)c->sm_count * per_sm;
     if (g > kMaxGrid) g = kMaxGrid;
-    if (g > num_chunks) g = num_chunks;
+    if (g > units) g = units;
     if (g < 1) g = 1;
     return (int)g;
 }
@@ -127,31 +148,47 @@ StepParams make_step_params(gxpo_ctx* c, int which_grad, int in_sel, int out_sel
     p.snapshot = snapshot;
     p.want_norm = want_norm;
     const gxpo_opt_cfg& o = c->opt;
-    p.lr = o.lr;
+    p.lr = (float)o.lr;
     if (o.kind == GXPO_OPT_ADAMW) {
-        // constants are formed in double from the float hyper-parameters, rounded once
+        // constants are formed in double from the double hyper-parameters, rounded once
         const double t = (double)c->t_opt;   // already incremented for this step
-        const double b1 = (double)o.beta1, b2 = (double)o.beta2, lr = (double)o.lr;
-        p.beta1 = o.beta1;
-        p.beta2 = o.beta2;
+        const double b1 = o.beta1, b2 = o.beta2, lr = o.lr;
+        p.beta1 = (float)b1;
+        p.beta2 = (float)b2;
         p.omb1 = (float)(1.0 - b1);
         p.omb2 = (float)(1.0 - b2);
-        p.eps = o.eps;
-        p.decay = (float)(1.0 - lr * (double)o.weight_decay);
+        p.eps = (float)o.eps;
+        p.decay = (float)(1.0 - lr * o.weight_decay);
         p.step_size = (float)(lr / (1.0 - std::pow(b1, t)));
         p.inv_sqrt_bc2 = (float)(1.0 / std::sqrt(1.0 - std::pow(b2, t)));
     }
     return p;
 }
 
-template <bool ADAMW, typename G>
-void launch_step_t(int variant, int grid, cudaStream_t s, const TensorDesc* descs,
-                   const ChunkRef* chunks, long long num_chunks, const TensorDesc& flat,
-                   const StepParams& p, double* partials, unsigned* ticket, double* sumsq) {
-    if (variant == 1)
-        step_kernel<ADAMW, G, 4><<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, partials, ticket, sumsq);
-    else
-        step_kernel<ADAMW, G, 8><<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, partials, ticket, sumsq);
+typedef void (*StepFn)(const TensorDesc*, const ChunkRef*, long long, TensorDesc, StepParams, int,
+                       double*, unsigned*, double*);
+typedef void (*ExtrapFn)(const TensorDesc*, const ChunkRef*, long long, TensorDesc, ExtrapParams, int);
+typedef void (*FusedFn)(const TensorDesc*, const ChunkRef*, long long, TensorDesc, FusedParams, int);
+
+StepFn pick_step(bool adamw, bool bf16, int variant) {
+    if (variant == 1) {
+        if (adamw) return bf16 ? step_kernel<true, uint16_t, 4> : step_kernel<true, float, 4>;
+        return bf16 ? step_kernel<false, uint16_t, 4> : step_kernel<false, float, 4>;
+    }
+    if (adamw) return bf16 ? step_kernel<true, uint16_t, 8> : step_kernel<true, float, 8>;
+    return bf16 ? step_kernel<false, uint16_t, 8> : step_kernel<false, float, 8>;
+}
+ExtrapFn pick_extrap(bool bf16, int variant) {
+    if (variant == 1) return bf16 ? extrap_kernel<uint16_t, 4> : extrap_kernel<float, 4>;
+    return bf16 ? extrap_kernel<uint16_t, 8> : extrap_kernel<float, 8>;
+}
+FusedFn pick_fused(bool adamw, bool bf16, int variant) {
+    if (variant == 1) {
+        if (adamw) return bf16 ? fused_kernel<true, uint16_t, 4> : fused_kernel<true, float, 4>;
+        return bf16 ? fused_kernel<false, uint16_t, 4> : fused_kernel<false, float, 4>;
+    }
+    if (adamw) return bf16 ? fused_kernel<true, uint16_t, 8> : fused_kernel<true, float, 8>;
+    return bf16 ? fused_kernel<false, uint16_t, 8> : fused_kernel<false, float, 8>;
 }
 
 // Launch one OptimStep sweep over either the bound list (chunks != null) or one
@@ -164,12 +201,9 @@ gxpo_status launch_step(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, co
         return GXPO_OK;
     }
     const bool adamw = c->opt.kind == GXPO_OPT_ADAMW;
-    const int grid = grid_for(c, num_chunks, adamw ? 4 : 6);
-    const bool bf16 = c->grad_dtype == GXPO_BF16;
-    if (adamw && bf16) launch_step_t<true, uint16_t>(c->variant, grid, s, descs, chunks, num_chunks, flat, p, c->d_partials, c->d_ticket, sumsq);
-    else if (adamw) launch_step_t<true, float>(c->variant, grid, s, descs, chunks, num_chunks, flat, p, c->d_partials, c->d_ticket, sumsq);
-    else if (bf16) launch_step_t<false, uint16_t>(c->variant, grid, s, descs, chunks, num_chunks, flat, p, c->d_partials, c->d_ticket, sumsq);
-    else launch_step_t<false, float>(c->variant, grid, s, descs, chunks, num_chunks, flat, p, c->d_partials, c->d_ticket, sumsq);
+    StepFn fn = pick_step(adamw, c->grad_dtype == GXPO_BF16, c->variant);
+    const int grid = grid_for(c, (const void*)fn, num_chunks << c->unit_shift, kDefaultCtasStep);
+    fn<<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, c->unit_shift, c->d_partials, c->d_ticket, sumsq);
     c->launches += 1;
     CUDA_TRY(c, cudaGetLastError());
     return GXPO_OK;
@@ -178,15 +212,20 @@ gxpo_status launch_step(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, co
 gxpo_status launch_extrap(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
                           long long num_chunks, const TensorDesc& flat, const ExtrapParams& p) {
     if (num_chunks <= 0) return GXPO_OK;
-    const int grid = grid_for(c, num_chunks, 6);
-    const bool bf16 = c->grad_dtype == GXPO_BF16;
-    if (c->variant == 1) {
-        if (bf16) extrap_kernel<uint16_t, 4><<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p);
-        else extrap_kernel<float, 4><<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p);
-    } else {
-        if (bf16) extrap_kernel<uint16_t, 8><<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p);
-        else extrap_kernel<float, 8><<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p);
-    }
+    ExtrapFn fn = pick_extrap(c->grad_dtype == GXPO_BF16, c->variant);
+    const int grid = grid_for(c, (const void*)fn, num_chunks << c->unit_shift, kDefaultCtasExtrap);
+    fn<<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, c->unit_shift);
+    c->launches += 1;
+    CUDA_TRY(c, cudaGetLastError());
+    return GXPO_OK;
+}
+
+gxpo_status launch_fused(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
+                         long long num_chunks, const TensorDesc& flat, const FusedParams& p) {
+    if (num_chunks <= 0) return GXPO_OK;
+    FusedFn fn = pick_fused(c->opt.kind == GXPO_OPT_ADAMW, c->grad_dtype == GXPO_BF16, c->variant);
+    const int grid = grid_for(c, (const void*)fn, num_chunks << c->unit_shift, kDefaultCtasFused);
+    fn<<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, c->unit_shift);
     c->launches += 1;
     CUDA_TRY(c, cudaGetLastError());
     return GXPO_OK;
@@ -288,11 +327,11 @@ void gxpo_default_cfg(gxpo_cfg* cfg, gxpo_opt_cfg* opt) {
     }
     if (opt) {
         opt->kind = GXPO_OPT_ADAMW;
-        opt->lr = 1e-7f;
-        opt->beta1 = 0.9f;
-        opt->beta2 = 0.999f;
-        opt->eps = 1e-8f;
-        opt->weight_decay = 0.01f;
+        opt->lr = 1e-7;
+        opt->beta1 = 0.9;
+        opt->beta2 = 0.999;
+        opt->eps = 1e-8;
+        opt->weight_decay = 0.01;
     }
 }
 
@@ -309,6 +348,7 @@ gxpo_status gxpo_create(const gxpo_cfg* cfg, const gxpo_opt_cfg* opt, int grad_d
     c->opt = *opt;
     c->grad_dtype = grad_dtype;
     c->variant = 2;
+    c->unit_shift = kDefaultUnitShift;
     c->s_star = -1;
     c->phase = IDLE;
     cudaError_t e = cudaGetDevice(&c->device);
@@ -455,6 +495,21 @@ gxpo_status gxpo_extrapolate(gxpo_ctx* c, void* stream) {
     return GXPO_OK;
 }
 
+gxpo_status gxpo_probe_extrapolate(gxpo_ctx* c, void* stream) {
+    if (!c) return GXPO_ERR_INVALID_ARG;
+    if (c->phase != PROBED0) return fail(c, GXPO_ERR_STATE, "fused probe+extrapolate must follow probe step 0");
+    const TensorDesc none = {};
+    const int place = c->cfg.placement;
+    c->t_opt += 1;
+    FusedParams p;
+    p.step = (place == GXPO_PLACE_PINGPONG) ? make_step_params(c, 1, 1, 1, 0, 0) : make_step_params(c, 1, 0, 0, 0, 0);
+    p.ex = make_extrap_params(c, place);
+    gxpo_status st = launch_fused(c, (cudaStream_t)stream, c->d_descs, c->d_chunks, c->num_chunks, none, p);
+    if (st != GXPO_OK) { c->t_opt -= 1; return st; }
+    c->phase = EXTRAPOLATED;
+    return GXPO_OK;
+}
+
 gxpo_status gxpo_slow_step(gxpo_ctx* c, void* stream) {
     if (!c) return GXPO_ERR_INVALID_ARG;
     if (c->phase != EXTRAPOLATED) return fail(c, GXPO_ERR_STATE, "slow step must follow extrapolate");
@@ -516,12 +571,17 @@ const char* gxpo_status_string(gxpo_status s) {
     return "unknown status";
 }
 
-gxpo_status gxpo_tune(gxpo_ctx* c, int ctas_per_sm, int variant) {
+gxpo_status gxpo_tune(gxpo_ctx* c, int ctas_per_sm, int variant, int unit_tiles) {
     if (!c) return GXPO_ERR_INVALID_ARG;
     if (ctas_per_sm < 0 || ctas_per_sm > 16) return fail(c, GXPO_ERR_INVALID_ARG, "ctas_per_sm must be in [0, 16]");
     if (variant < 0 || variant > 2) return fail(c, GXPO_ERR_INVALID_ARG, "variant must be 0, 1 or 2");
+    int ush = -1;
+    if (unit_tiles == 0) ush = kDefaultUnitShift;
+    for (int k = 0; k <= 4; ++k) if (unit_tiles == (kTilesPerChunk >> k)) ush = k;
+    if (ush < 0) return fail(c, GXPO_ERR_INVALID_ARG, "unit_tiles must be 0, 1, 2, 4, 8 or 16");
     c->ctas_per_sm = ctas_per_sm;
     c->variant = variant == 0 ? 2 : variant;
+    c->unit_shift = ush;
     return GXPO_OK;
 }
 
@@ -631,9 +691,10 @@ gxpo_status gxpo_step_host(gxpo_ctx* c, const gxpo_tensor* list, int count, long
                 rs = launch_step(c, s, nullptr, nullptr, nch, d, make_step_params(c, 0, 0, 1, 0, 0), c->d_sumsq);
                 if (rs != GXPO_OK) return rs;
                 c->t_opt = t_opt0 + 2;
-                rs = launch_step(c, s, nullptr, nullptr, nch, d, make_step_params(c, 1, 1, 1, 0, 0), c->d_sumsq);
-                if (rs != GXPO_OK) return rs;
-                rs = launch_extrap(c, s, nullptr, nullptr, nch, d, make_extrap_params(c, GXPO_PLACE_PINGPONG));
+                FusedParams fp;
+                fp.step = make_step_params(c, 1, 1, 1, 0, 0);
+                fp.ex = make_extrap_params(c, GXPO_PLACE_PINGPONG);
+                rs = launch_fused(c, s, nullptr, nullptr, nch, d, fp);
                 if (rs != GXPO_OK) return rs;
                 c->t_opt = t_opt0 + 3;
                 rs = launch_step(c, s, nullptr, nullptr, nch, d, make_step_params(c, 2, 0, 0, 0, 1), st.piece_sumsq + 1);

@@ -36,5 +36,5 @@ def test_status_strings_and_defaults_need_no_gpu():
     cfg, opt = b.default_cfg()
     assert (cfg.K, cfg.window, cfg.min_history, cfg.std_ddof, cfg.placement) == (5, 20, 2, 0, 0)
     assert abs(cfg.alpha - 0.5) < 1e-7 and abs(cfg.tau - 0.5) < 1e-15 and abs(cfg.delta - 1e-8) < 1e-12
-    assert opt.kind == b.OPT_ADAMW and abs(opt.lr - 1e-7) < 1e-12
+    assert opt.kind == b.OPT_ADAMW and opt.lr == 1e-7 and opt.beta2 == 0.999
     assert b._lib.gxpo_status_string(b.ERR_STATE).decode() == "call out of order"

@@ -199,7 +199,7 @@ def test_call_order_and_argument_checks():
     res = ctx.gate_update()
     assert res.t == 1 and ctx.optimizer_steps() == 3
     with pytest.raises(b.GxpoError) as e:
-        ctx.tune(99, 0)
+        ctx.tune(99, 0, 0)
     assert e.value.status == b.ERR_INVALID_ARG
     assert "ctas_per_sm" in str(e.value)
     torch.cuda.synchronize()
