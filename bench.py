@@ -3,7 +3,8 @@
 
 A "step" is one whole active step of Algorithm 1's parameter-space update over
 the workload's tensor list: probe step 0, probe step 1, extrapolate + reposition,
-slow step with the in-sweep norm, gate update (4 sweeps + 1 tiny kernel).  The
+slow step with the in-sweep norm, gate update (3 sweeps + 1 tiny kernel by default:
+probe step 1 and the extrapolation share one sweep; --unfused makes it 4).  The
 three gradient buffers are synthetic and already resident.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
@@ -83,13 +84,21 @@ def measured_peak_gbs():
 
 
 def recorded_traffic_per_param():
-    """DRAM bytes per parameter of the dominant kernel from the committed ncu summary."""
-    path = os.path.join(ROOT, "profiles", "step_kernel_traffic.json")
+    """DRAM bytes per parameter of the dominant kernel, from the committed ncu summary.
+    The summary records the hash of the kernel source it was taken from; once that
+    source has changed the counters no longer describe the kernel and None is returned."""
+    import hashlib
+    import re
+    summary = os.path.join(ROOT, "profiles", "step_kernel_adamw_bf16_flat134m.txt")
+    source = os.path.join(ROOT, "paper_2605_06755_b200", "csrc", "gxpo_kernels.cuh")
     try:
-        with open(path) as f:
-            return float(json.load(f)["dram_bytes_per_param"])
+        text = open(summary).read()
+        want = re.search(r"^kernel_source_sha256:\s*([0-9a-f]{64})", text, re.M).group(1)
+        per_param = float(re.search(r"^dram_bytes_per_param:\s*([0-9.]+)", text, re.M).group(1))
+        have = hashlib.sha256(open(source, "rb").read()).hexdigest()
     except Exception:
         return None
+    return per_param if have == want else None
 
 
 # ----------------------------------------------------------------------------
