@@ -219,6 +219,47 @@ gxpo_status gxpo_step_host(gxpo_ctx* ctx, const gxpo_tensor* list, int count,
  * summation order of the norm changes. */
 gxpo_status gxpo_tune(gxpo_ctx* ctx, int ctas_per_sm, int variant, int unit_tiles);
 
+/* The slow correction for callers that must not allocate.  (The paper has no
+ * counterpart to this entry point: it is the same update as gxpo_slow_step, packaged
+ * differently.)
+ *
+ * Who needs it: a trainer that has handed all device memory to its own pool, or that
+ * runs with the GPU nearly full (a 7.6e9-parameter list occupies 167 of 180 GB), cannot
+ * rely on gxpo_create's cudaMalloc succeeding; code that runs inside another library's
+ * callback, or under a policy that forbids allocation after start-up, may not call it at
+ * all.  This function needs no context and calls no cudaMalloc, cudaFree or any other
+ * allocating routine: its reduction scratch is an array built into the library image
+ * (about 512 KB, resident on every GPU that loads the library until the process exits).
+ *
+ * What it does, for ONE flat buffer of n parameters, in place:
+ *     theta <- OptimStep(theta, g_slow)   (m, v updated for AdamW; may be NULL for GD)
+ *     *sumsq_dev <- sum(g_slow^2)         (float64; take the square root for the norm)
+ * theta, m, v, g_slow and sumsq_dev are DEVICE pointers owned by the caller; g_slow has
+ * dtype `grad_dtype`.  `t_opt` is the optimizer's step count INCLUDING this step (the
+ * third step of the first active step has t_opt = 3); it only matters for AdamW's bias
+ * correction.  The work is enqueued on `stream` and not waited for.
+ *
+ * Limits and sharing:
+ *   - n <= GXPO_NOALLOC_MAX_PARAMS; larger n is rejected with GXPO_ERR_INVALID_ARG and a
+ *     message saying so.  Split a larger buffer and add the sums.
+ *   - The partial sums are taken per 32768-parameter chunk and added in chunk order, so
+ *     the result depends only on the data, not on the launch shape.  It can differ from
+ *     gxpo_slow_step's sum in the last bits (different grouping).
+ *   - All calls on one GPU share the one scratch array, whatever the stream or thread.
+ *     Calls that overlap on the GPU race on it and give wrong sums: order them (same
+ *     stream, or events).  Each call resets the part of the scratch that must start at
+ *     zero, so the previous call's contents never leak into the next.
+ *   - The first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress) with that device current; make that first call outside any
+ *     stream capture.
+ * Errors: a status code as everywhere else; if `errbuf` is not NULL, a description of
+ * the failure is written there (at most errbuf_len bytes, NUL-terminated). */
+#define GXPO_NOALLOC_MAX_PARAMS 2147483648LL
+gxpo_status gxpo_slow_step_noalloc(float* theta, float* m, float* v, const void* g_slow,
+                                   long long n, int grad_dtype, const gxpo_opt_cfg* opt,
+                                   long long t_opt, double* sumsq_dev, void* stream,
+                                   char* errbuf, size_t errbuf_len);
+
 /* Number of kernels this context has launched so far. */
 long long gxpo_launch_count(const gxpo_ctx* ctx);
 

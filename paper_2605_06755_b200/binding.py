@@ -85,6 +85,9 @@ _sigs = {
                                              ctypes.c_int, ctypes.c_float, ctypes.c_float,
                                              ctypes.c_float, _vp, _vp, _vp]),
     "gxpo_quad_scratch_bytes": (ctypes.c_size_t, []),
+    "gxpo_slow_step_noalloc": (ctypes.c_int, [_vp, _vp, _vp, _vp, ctypes.c_longlong, ctypes.c_int,
+                                              ctypes.POINTER(OptCfg), ctypes.c_longlong, _vp, _vp,
+                                              ctypes.c_char_p, ctypes.c_size_t]),
 }
 for _name, (_res, _args) in _sigs.items():
     _f = getattr(_lib, _name)
@@ -271,6 +274,22 @@ def quad_active_step(theta_ptr, a_ptr, b_ptr, n, lr, K, alpha, delta, den_eps, s
                                     sumsq_ptr, scratch_ptr, _stream_ptr(stream))
     if st != OK:
         raise GxpoError(st, "gxpo_quad_active_step")
+
+
+NOALLOC_MAX_PARAMS = 2147483648
+
+
+def slow_step_noalloc(theta_ptr, m_ptr, v_ptr, g_slow_ptr, n, grad_dtype, opt: OptCfg, t_opt,
+                      sumsq_ptr, stream=None):
+    """gxpo_slow_step_noalloc: the slow correction on one flat buffer, in place, with
+    sum(g_slow^2) written to the device double at `sumsq_ptr`.  Needs no Context and
+    allocates nothing; see include/gxpo.h for the size limit and the sharing rules."""
+    err = ctypes.create_string_buffer(512)
+    st = _lib.gxpo_slow_step_noalloc(theta_ptr or None, m_ptr or None, v_ptr or None,
+                                     g_slow_ptr or None, n, grad_dtype, ctypes.byref(opt), t_opt,
+                                     sumsq_ptr or None, _stream_ptr(stream), err, len(err))
+    if st != OK:
+        raise GxpoError(st, err.value.decode())
 
 
 def tensor_ptrs(theta, work, m, v, g0, g1, g_slow) -> TensorPtrs:

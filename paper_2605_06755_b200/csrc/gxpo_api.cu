@@ -7,6 +7,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -765,3 +766,184 @@ gxpo_status gxpo_quad_active_step(float* theta, const float* a, const float* b, 
 }
 
 }  // extern "C"
+
+// ---- allocation-free slow step ----------------------------------------------------
+// Everything this entry point needs lives in this file: the scratch array, the variant
+// of the OptimStep sweep that writes one partial sum per chunk into it, the per-device
+// set-up that turns the array's name into a device address, and the entry point.
+namespace {
+
+constexpr long long kNoAllocMaxChunks = GXPO_NOALLOC_MAX_PARAMS / kChunk;   // 65536
+constexpr size_t kNoAllocPartialBytes = (size_t)kNoAllocMaxChunks * sizeof(double);
+constexpr int kNoAllocMaxDevices = 64;
+
+// One float64 partial per 32768-element chunk (512 KB), then the ticket counter in a
+// 256-byte cell of its own.  Held by every device that loads the library, until exit.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocPartialBytes + 256];
+
+// The OptimStep sweep over one flat buffer with sum(g^2) reduced per chunk: each chunk's
+// partial lands in its own slot and the last CTA to finish adds the slots in index
+// order, so the sum depends on n alone and not on how many CTAs ran.
+template <bool ADAMW, typename G>
+__global__ void __launch_bounds__(kThreads)
+step_flat_perchunk_kernel(TensorDesc d, long long num_chunks, StepParams p, double* partials,
+                          unsigned* ticket, double* sumsq_out) {
+    __shared__ double red[8];
+    for (long long c = blockIdx.x; c < num_chunks; c += gridDim.x) {
+        const long long off = c * kChunk;
+        const long long rem = d.n - off;
+        const int len = rem < kChunk ? (int)rem : kChunk;
+        float* th = d.theta + off;
+        float* m = ADAMW ? d.m + off : nullptr;
+        float* v = ADAMW ? d.v + off : nullptr;
+        const G* g = reinterpret_cast<const G*>(d.g[2]) + off;
+        const bool vec = aligned32(th) && aligned32(g) && (!ADAMW || (aligned32(m) && aligned32(v)));
+        double acc = 0.0;
+        if (vec) step_chunk_vec<ADAMW, G, 8>(th, th, nullptr, m, v, g, len, p, acc);
+        else     step_chunk_scalar<ADAMW, G>(th, th, nullptr, m, v, g, len, p, acc);
+        const double tot = block_sum(acc, red);
+        if (threadIdx.x == 0) partials[c] = tot;
+    }
+    __shared__ bool is_last;
+    if (threadIdx.x == 0) {
+        __threadfence();
+        is_last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (is_last) {
+        __threadfence();
+        double s = 0.0;
+        for (long long i = threadIdx.x; i < num_chunks; i += kThreads) s += __ldcg(partials + i);
+        s = block_sum(s, red);
+        if (threadIdx.x == 0) {
+            *sumsq_out = s;
+            *ticket = 0u;
+        }
+    }
+}
+
+struct NoAllocDevice {
+    bool ready;
+    unsigned char* scratch;    // device address of g_noalloc_scratch on this device
+    int sm_count;
+};
+NoAllocDevice g_noalloc_dev[kNoAllocMaxDevices];
+std::mutex g_noalloc_mutex;
+
+gxpo_status noalloc_fail(char* buf, size_t len, gxpo_status s, const char* fmt, ...) {
+    if (buf && len > 0) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(buf, len, fmt, ap);
+        va_end(ap);
+    }
+    return s;
+}
+
+}  // namespace
+
+extern "C" gxpo_status gxpo_slow_step_noalloc(float* theta, float* m, float* v, const void* g_slow,
+                                              long long n, int grad_dtype, const gxpo_opt_cfg* opt,
+                                              long long t_opt, double* sumsq_dev, void* stream,
+                                              char* errbuf, size_t errbuf_len) {
+    if (errbuf && errbuf_len > 0) errbuf[0] = '\0';
+    if (!opt || !sumsq_dev) return noalloc_fail(errbuf, errbuf_len, GXPO_ERR_INVALID_ARG, "opt and sumsq_dev must not be null");
+    if (grad_dtype != GXPO_F32 && grad_dtype != GXPO_BF16) return noalloc_fail(errbuf, errbuf_len, GXPO_ERR_INVALID_ARG, "unknown gradient dtype %d", grad_dtype);
+    if (opt->kind != GXPO_OPT_GD && opt->kind != GXPO_OPT_ADAMW) return noalloc_fail(errbuf, errbuf_len, GXPO_ERR_INVALID_ARG, "unknown optimizer kind %d", opt->kind);
+    const bool adamw = opt->kind == GXPO_OPT_ADAMW;
+    if (!std::isfinite(opt->lr)) return noalloc_fail(errbuf, errbuf_len, GXPO_ERR_INVALID_ARG, "lr is not finite");
+    if (adamw) {
+        if (!(opt->beta1 >= 0.0 && opt->beta1 < 1.0) || !(opt->beta2 >= 0.0 && opt->beta2 < 1.0))
+            return noalloc_fail(errbuf, errbuf_len, GXPO_ERR_INVALID_ARG, "betas must be in [0, 1)");
+        if (!(opt->eps >= 0.0) || !std::isfinite(opt->eps) || !std::isfinite(opt->weight_decay))
+            return noalloc_fail(errbuf, errbuf_len, GXPO_ERR_INVALID_ARG, "eps must be finite and >= 0, weight_decay finite");
+        if (t_opt < 1) return noalloc_fail(errbuf, errbuf_len, GXPO_ERR_INVALID_ARG, "t_opt counts this step and must be >= 1, got %lld", t_opt);
+    }
+    if (n < 0) return noalloc_fail(errbuf, errbuf_len, GXPO_ERR_INVALID_ARG, "n < 0");
+    if (n > GXPO_NOALLOC_MAX_PARAMS)
+        return noalloc_fail(errbuf, errbuf_len, GXPO_ERR_INVALID_ARG,
+                            "n = %lld exceeds GXPO_NOALLOC_MAX_PARAMS = %lld (the built-in scratch holds one partial sum per %d parameters); "
+                            "split the buffer and add the sums, or use a context", n, (long long)GXPO_NOALLOC_MAX_PARAMS, kChunk);
+    if (((uintptr_t)sumsq_dev) & 7u) return noalloc_fail(errbuf, errbuf_len, GXPO_ERR_ALIGNMENT, "sumsq_dev must be 8-byte aligned");
+    if (n > 0) {
+        if (!theta || !g_slow || (adamw && (!m || !v)))
+            return noalloc_fail(errbuf, errbuf_len, GXPO_ERR_INVALID_ARG, "null theta/m/v/g_slow pointer");
+        const uintptr_t gmask = (grad_dtype == GXPO_BF16) ? 1u : 3u;
+        if ((((uintptr_t)theta) & 3u) || (((uintptr_t)m) & 3u) || (((uintptr_t)v) & 3u) || (((uintptr_t)g_slow) & gmask))
+            return noalloc_fail(errbuf, errbuf_len, GXPO_ERR_ALIGNMENT, "a pointer is not aligned to its element size");
+    }
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e;
+
+    // Per-device set-up, first call on each device: in host code the array's name is only
+    // a handle, so ask the runtime for its address on the current device and keep it.
+    int dev = -1;
+    e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return noalloc_fail(errbuf, errbuf_len, GXPO_ERR_CUDA, "cudaGetDevice failed: %s", cudaGetErrorString(e));
+    if (dev < 0 || dev >= kNoAllocMaxDevices) return noalloc_fail(errbuf, errbuf_len, GXPO_ERR_INVALID_ARG, "device ordinal %d out of range", dev);
+    NoAllocDevice nd;
+    {
+        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+        if (!g_noalloc_dev[dev].ready) {
+            void* ptr = nullptr;
+            e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+            if (e != cudaSuccess || !ptr)
+                return noalloc_fail(errbuf, errbuf_len, GXPO_ERR_CUDA, "cudaGetSymbolAddress failed: %s", cudaGetErrorString(e));
+            int sms = 0;
+            e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+            if (e != cudaSuccess || sms < 1)
+                return noalloc_fail(errbuf, errbuf_len, GXPO_ERR_CUDA, "cudaDeviceGetAttribute failed: %s", cudaGetErrorString(e));
+            g_noalloc_dev[dev].scratch = static_cast<unsigned char*>(ptr);
+            g_noalloc_dev[dev].sm_count = sms;
+            g_noalloc_dev[dev].ready = true;
+        }
+        nd = g_noalloc_dev[dev];
+    }
+    double* partials = reinterpret_cast<double*>(nd.scratch);
+    unsigned* ticket = reinterpret_cast<unsigned*>(nd.scratch + kNoAllocPartialBytes);
+
+    if (n == 0) {
+        e = cudaMemsetAsync(sumsq_dev, 0, sizeof(double), s);
+        if (e != cudaSuccess) return noalloc_fail(errbuf, errbuf_len, GXPO_ERR_CUDA, "cudaMemsetAsync failed: %s", cudaGetErrorString(e));
+        return GXPO_OK;
+    }
+    // The array keeps whatever the last call left: the counter must start at zero (an
+    // earlier call that failed to launch could have left it mid-count); the partial slots
+    // need no clearing because every slot that is read is written first.
+    e = cudaMemsetAsync(ticket, 0, sizeof(unsigned), s);
+    if (e != cudaSuccess) return noalloc_fail(errbuf, errbuf_len, GXPO_ERR_CUDA, "cudaMemsetAsync failed: %s", cudaGetErrorString(e));
+
+    StepParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.which_grad = 2;
+    p.want_norm = 1;
+    p.lr = (float)opt->lr;
+    if (adamw) {
+        const double t = (double)t_opt, b1 = opt->beta1, b2 = opt->beta2, lr = opt->lr;
+        p.beta1 = (float)b1;
+        p.beta2 = (float)b2;
+        p.omb1 = (float)(1.0 - b1);
+        p.omb2 = (float)(1.0 - b2);
+        p.eps = (float)opt->eps;
+        p.decay = (float)(1.0 - lr * opt->weight_decay);
+        p.step_size = (float)(lr / (1.0 - std::pow(b1, t)));
+        p.inv_sqrt_bc2 = (float)(1.0 / std::sqrt(1.0 - std::pow(b2, t)));
+    }
+    TensorDesc d;
+    std::memset(&d, 0, sizeof(d));
+    d.theta = theta; d.m = m; d.v = v; d.g[2] = g_slow; d.n = n;
+    const long long num_chunks = (n + kChunk - 1) / kChunk;
+    long long grid = (long long)nd.sm_count * kDefaultCtasStep;
+    if (grid > num_chunks) grid = num_chunks;
+    const bool bf16 = grad_dtype == GXPO_BF16;
+    if (adamw) {
+        if (bf16) step_flat_perchunk_kernel<true, uint16_t><<<(int)grid, kThreads, 0, s>>>(d, num_chunks, p, partials, ticket, sumsq_dev);
+        else      step_flat_perchunk_kernel<true, float><<<(int)grid, kThreads, 0, s>>>(d, num_chunks, p, partials, ticket, sumsq_dev);
+    } else {
+        if (bf16) step_flat_perchunk_kernel<false, uint16_t><<<(int)grid, kThreads, 0, s>>>(d, num_chunks, p, partials, ticket, sumsq_dev);
+        else      step_flat_perchunk_kernel<false, float><<<(int)grid, kThreads, 0, s>>>(d, num_chunks, p, partials, ticket, sumsq_dev);
+    }
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return noalloc_fail(errbuf, errbuf_len, GXPO_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+    return GXPO_OK;
+}
