@@ -234,6 +234,24 @@ def build_device_workload(torch, b, shapes, seed, alias_gslow):
     return d, ptrs, (theta, work, m, v, g0, g1, gs)
 
 
+def plan_workload(args, free_bytes, margin=6 << 30):
+    """Shapes of the workload and whether g_slow has to share g0's buffer (legal: g0 is
+    dead once the extrapolation has run) so that 22 -> 20 bytes per parameter fit into
+    the free device memory; as a last resort the decoder depth is reduced, and the
+    description says so."""
+    shapes, desc = workload_shapes(args)
+    d = sum(k for _, k in shapes)
+    alias = 22 * d + margin > free_bytes
+    while (20 if alias else 22) * d + margin > free_bytes and args.workload in ("qwen25_7b", "llama31_8b"):
+        args.layers = (args.layers or (28 if args.workload == "qwen25_7b" else 32)) - 1
+        if args.layers < 1:
+            raise SystemExit("not enough free device memory for even one decoder layer")
+        shapes, desc = workload_shapes(args)
+        desc += f" (reduced to {args.layers} layers: not enough free device memory)"
+        d = sum(k for _, k in shapes)
+    return shapes, desc, alias
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -253,18 +271,8 @@ def run_ours(args):
     props = torch.cuda.get_device_properties(local)
     stream = torch.cuda.current_stream()
 
-    shapes, desc = workload_shapes(args)
-    d = sum(k for _, k in shapes)
     free, total = torch.cuda.mem_get_info()
-    margin = 6 << 30
-    alias = False
-    if 22 * d + margin > free:
-        alias = True                      # g_slow reuses g0's buffer (g0 is dead after extrapolate)
-    while (20 if alias else 22) * d + margin > free and args.workload in ("qwen25_7b", "llama31_8b"):
-        args.layers = (args.layers or (28 if args.workload == "qwen25_7b" else 32)) - 1
-        shapes, desc = workload_shapes(args)
-        desc += f" (reduced to {args.layers} layers: not enough free device memory)"
-        d = sum(k for _, k in shapes)
+    shapes, desc, alias = plan_workload(args, free)
     d, ptrs, keep = build_device_workload(torch, b, shapes, 1000 + rank, alias)
     sumsq = torch.zeros(1, dtype=torch.float64, device="cuda")
 

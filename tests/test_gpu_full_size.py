@@ -1,0 +1,246 @@
+"""Parity at the full sizes of the benchmark configurations, in the launch
+configuration bench.py times (default grid and access width, probe step 1 fused
+with the extrapolation): the flat 1.54e9-parameter buffer, the Qwen2.5-7B-shaped
+list (7.6e9) and the 64-step gate stream on the Llama-3.1-8B-shaped list (8.0e9).
+
+The update is per-coordinate, so the oracle run on a window of the inputs IS the
+full run restricted to that window: windows are copied to the host before the step
+(the same bits the kernels read), run through the CPU oracle, and compared element
+by element afterwards.  Windows cover tensor starts and ends, chunk boundaries,
+whole small tensors and the ragged tail.  The one global quantity, ||g_slow||, is
+compared with the oracle's sum over the whole buffer where that takes seconds
+(1.54e9) and with a float64 library reduction otherwise; the library reduction is
+itself tied to the oracle on sampled tensors."""
+import argparse
+import gc
+import math
+
+import numpy as np
+import pytest
+
+from oracle import gxpo_oracle as ora
+from tests import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+WIN = 40000        # elements per window: a 32768-element chunk boundary falls inside most of them
+
+
+def _setup(workload, lr, K=5, alpha=0.5):
+    """Device workload exactly as bench.py builds it."""
+    import torch
+
+    import bench
+    from paper_2605_06755_b200 import binding as b
+    gc.collect()
+    torch.cuda.empty_cache()
+    args = argparse.Namespace(workload=workload, layers=0, params=0)
+    free, _ = torch.cuda.mem_get_info()
+    shapes, desc, alias = bench.plan_workload(args, free)
+    d, ptrs, keep = bench.build_device_workload(torch, b, shapes, 2026, alias)
+    cfg, opt = b.make_cfg(K=K, alpha=alpha, lr=lr)
+    ctx = b.Context(cfg, opt, b.BF16)
+    ctx.bind(ptrs)
+    return b, ctx, cfg, opt, shapes, desc, alias, d, keep
+
+
+def _windows(shapes, picks):
+    """Global [lo, hi) ranges in the concatenated parameter space.  `picks` is a list of
+    (tensor index, 'head' | 'tail' | 'all' | 'chunk' | 'mid')."""
+    starts, acc = [], 0
+    for _, n in shapes:
+        starts.append(acc)
+        acc += n
+    out = []
+    for t, where in picks:
+        s, n = starts[t], shapes[t][1]
+        if where == "all" or n <= WIN:
+            lo, hi = s, s + n
+        elif where == "head":
+            lo, hi = s, s + WIN
+        elif where == "tail":
+            lo, hi = s + n - WIN, s + n
+        elif where == "chunk":                    # straddles an interior 32768-element chunk boundary
+            c = (n // 32768 // 2) * 32768
+            lo, hi = s + c - WIN // 2, s + c + WIN // 2
+        else:
+            lo, hi = s + n // 3, s + n // 3 + WIN
+        out.append((max(lo, s), min(hi, s + n)))
+    return out
+
+
+def _grab(keep, lo, hi):
+    """Host copies of one window of theta, m, v, g0, g1, g_slow (float64, exact)."""
+    theta, work, m, v, g0, g1, gs = keep
+    f = lambda t: gu.to_host_f64(t[lo:hi])
+    return dict(theta=f(theta), m=f(m), v=f(v), g0=f(g0), g1=f(g1), gs=f(gs))
+
+
+def _device_sumsq_f64(t, block=1 << 27):
+    """sum(x^2) by a float64 library reduction on the device, in bounded blocks."""
+    import torch
+    tot = 0.0
+    for s in range(0, t.numel(), block):
+        x = t[s:s + block].double()
+        tot += float(torch.dot(x, x).item())
+    return tot
+
+
+def _check_window(keep, lo, hi, st, scale, theta0, theta2, alpha, what, rtol=2e-6):
+    theta, work, m, v = keep[:4]
+    sat = ~np.isfinite(scale) | (np.abs(scale) > 1e30)
+    slack = gu.displacement_slack(theta0, theta2, scale, alpha)
+    nsat = gu.assert_close(gu.to_host_f64(theta[lo:hi]), st.theta, what + " theta", rtol=rtol,
+                           saturated=sat, extra_abs=slack)
+    gu.assert_close(gu.to_host_f64(m[lo:hi]), st.m, what + " m")
+    gu.assert_close(gu.to_host_f64(v[lo:hi]), st.v, what + " v")
+    return nsat
+
+
+def _one_active_step_vs_oracle(workload, lr, picks_fn, full_oracle_norm):
+    import torch
+    b, ctx, cfg, opt, shapes, desc, alias, d, keep = _setup(workload, lr)
+    assert "reduced" not in desc, desc           # the full size is the point of this test
+    gcfg, ocfg = gu.ora_cfgs(cfg, opt)
+    wins = _windows(shapes, picks_fn(shapes))
+    before = [_grab(keep, lo, hi) for lo, hi in wins]
+    gs = keep[6]
+    if full_oracle_norm:
+        sumsq, blk = 0.0, 1 << 26
+        for s in range(0, d, blk):
+            sumsq += ora.sum_squares(gu.to_host_f64(gs[s:s + blk]))
+        want_norm = math.sqrt(sumsq)
+    else:
+        want_norm = math.sqrt(_device_sumsq_f64(gs))
+        for lo, hi in wins[:3]:                   # tie the library reduction to the oracle
+            assert _device_sumsq_f64(gs[lo:hi]) == pytest.approx(
+                ora.sum_squares(gu.to_host_f64(gs[lo:hi])), rel=1e-12)
+    res = ctx.active_step(allow_nonfinite=True, fused=True)
+    torch.cuda.synchronize()
+    assert ctx.launch_count() == 4
+    assert res.norm == pytest.approx(want_norm, rel=gu.RTOL_NORM)
+    nsat = 0
+    for (lo, hi), w in zip(wins, before):
+        st = ora.State(w["theta"], ocfg, w["m"], w["v"])
+        grads = [w["g0"], w["g1"], w["gs"]]
+        trace = {}
+        ora.active_step(st, gcfg, lambda k, th: grads[k], round_f32=True, trace=trace)
+        nsat += _check_window(keep, lo, hi, st, trace["scale"], w["theta"], trace["theta2"], gcfg.alpha,
+                              f"{workload} [{lo},{hi})")
+    total = sum(hi - lo for lo, hi in wins)
+    assert nsat < 1e-3 * total                    # saturated scale factors are rare
+    ctx.close()
+    del keep
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("lr", [1e-7, 1e-3])
+def test_flat_1p54b_one_active_step(lr):
+    """Flat 1.54e9-parameter buffer, fp32 theta/m/v, bf16 gradients: one full active
+    step; windows at the start, at chunk boundaries, mid-buffer and the ragged tail;
+    the norm against the oracle's sum over all 1.54e9 gradients."""
+    def picks(shapes):
+        return [(0, "head"), (0, "chunk"), (0, "mid"), (0, "tail")]
+    _one_active_step_vs_oracle("flat_1p54b", lr, picks, full_oracle_norm=True)
+
+
+def _decoder_picks(shapes):
+    """Embedding head, every kind of tensor in the first and last layer (whole when
+    small), a mid-stack projection at a chunk boundary, final norm and the LM head's tail."""
+    names = [nm for nm, _ in shapes]
+    last = max(int(nm.split(".")[1]) for nm in names if nm.startswith("layers."))
+    picks = [(0, "head"), (0, "chunk")]
+    for i, nm in enumerate(names):
+        if nm.startswith("layers.0.") or nm.startswith(f"layers.{last}."):
+            picks.append((i, "tail" if nm.endswith("proj.weight") else "all"))
+        elif nm == f"layers.{last // 2}.down_proj.weight":
+            picks.append((i, "chunk"))
+    picks += [(len(names) - 2, "all"), (len(names) - 1, "head"), (len(names) - 1, "tail")]
+    return picks
+
+
+def test_qwen25_7b_list_one_active_step():
+    """The benchmark's own workload and hyper-parameters (lr = 1e-7): 339 tensors,
+    7,615,616,512 parameters, one active step."""
+    _one_active_step_vs_oracle("qwen25_7b", 1e-7, _decoder_picks, full_oracle_norm=False)
+
+
+def test_llama31_8b_list_64_step_gate_stream():
+    """64 training steps on the Llama-3.1-8B-shaped list; ||g_slow|| is scaled x1 for
+    steps 0..39 and x8 at step 40 (exact in bfloat16).  The library must fall back to
+    the single-pass step at exactly the oracle's step (s* = 41), and the sampled
+    windows must follow the oracle through all 41 active and 23 fallback steps."""
+    import torch
+    b, ctx, cfg, opt, shapes, desc, alias, d, keep = _setup("llama31_8b", 1e-3)
+    assert "reduced" not in desc, desc
+    gcfg, ocfg = gu.ora_cfgs(cfg, opt)
+    theta, work, m, v, g0, g1, gs = keep
+    # tame the ratios inside the windows only (64 chained steps would otherwise let a
+    # huge scale factor amplify last-ulp differences): g1 = g0 * u, u in [0.25, 1.25)
+    wins = _windows(shapes, _decoder_picks(shapes))
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(7)
+    for lo, hi in wins:
+        u = torch.rand(hi - lo, generator=gen, device="cuda") + 0.25
+        g1[lo:hi] = (g0[lo:hi].float() * u).to(torch.bfloat16)
+    states = []
+    for lo, hi in wins:
+        w = _grab(keep, lo, hi)
+        states.append((ora.State(w["theta"], ocfg, w["m"], w["v"]), [w["g0"], w["g1"], w["gs"]]))
+    # the norm stream the oracle's gate sees: the base norm by a float64 library
+    # reduction (tied to the oracle on windows), x8 at step 40
+    base = math.sqrt(_device_sumsq_f64(gs))
+    for lo, hi in wins[:3]:
+        assert _device_sumsq_f64(gs[lo:hi]) == pytest.approx(ora.sum_squares(gu.to_host_f64(gs[lo:hi])), rel=1e-12)
+    gate = ora.Gate(gcfg)
+    phases, t_active, t_fallback = [], [], []
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    for t in range(64):
+        mult = 8.0 if t == 40 else 1.0
+        lib_active, _, lib_t = ctx.gate_peek()
+        assert lib_t == t and lib_active == gate.active
+        ev[0].record()
+        if gate.active:
+            ctx.probe_step(0)
+            ctx.probe_extrapolate()
+            if mult != 1.0:
+                gs.mul_(mult)                     # the caller's third backward pass writes g_slow
+            ctx.slow_step()
+            res = ctx.gate_update()
+            if mult != 1.0:
+                gs.div_(mult)                     # g_slow may share g0's buffer: restore it
+            ev[1].record()
+            tripped, z, mu, sg = gate.update(base * mult)
+            assert bool(res.tripped) == tripped and res.s_star == gate.s_star
+            assert res.norm == pytest.approx(base * mult, rel=gu.RTOL_NORM)
+            for st, g in states:
+                gg = [g[0], g[1], g[2] * mult]
+                ora.active_step(st, gcfg, lambda k, th, gg=gg: gg[k], round_f32=True)
+            phases.append("a")
+        else:
+            ctx.probe_step(-1)
+            ev[1].record()
+            gate.fallback_tick()
+            for st, g in states:
+                ora.fallback_step(st, lambda k, th, g=g: g[k], round_f32=True)
+            phases.append("f")
+        torch.cuda.synchronize()
+        (t_active if phases[-1] == "a" else t_fallback).append(ev[0].elapsed_time(ev[1]))
+    assert gate.s_star == 41 and ctx.gate_peek()[1] == 41
+    assert "".join(phases) == "a" * 41 + "f" * 23
+    assert ctx.backward_passes() == ora.backward_budget(41, 64) == 3 * 41 + 23
+    assert ctx.optimizer_steps() == 3 * 41 + 23
+    for (lo, hi), (st, _) in zip(wins, states):
+        what = f"llama31_8b [{lo},{hi}) after 64 steps"
+        gu.assert_close(gu.to_host_f64(theta[lo:hi]), st.theta, what + " theta", rtol=2e-5)
+        gu.assert_close(gu.to_host_f64(m[lo:hi]), st.m, what + " m", rtol=5e-6)
+        gu.assert_close(gu.to_host_f64(v[lo:hi]), st.v, what + " v", rtol=5e-6)
+    # both paths were timed (milliseconds per step, steady state)
+    act = float(np.median(t_active[3:40])) if len(t_active) > 43 else float(np.median(t_active[3:]))
+    fb = float(np.median(t_fallback[1:]))
+    print(f"\nllama31_8b d={d}: active step {act:.1f} ms ({84 * d / act / 1e6:.0f} GB/s), "
+          f"fallback step {fb:.1f} ms ({26 * d / fb / 1e6:.0f} GB/s), g_slow aliases g0: {alias}")
+    assert fb < act
+    ctx.close()
+    del keep, theta, work, m, v, g0, g1, gs
+    torch.cuda.empty_cache()
