@@ -3,8 +3,10 @@
 
 A "step" is one whole active step of Algorithm 1's parameter-space update over
 the workload's tensor list: probe step 0, probe step 1, extrapolate + reposition,
-slow step with the in-sweep norm, gate update (3 sweeps + 1 tiny kernel by default:
-probe step 1 and the extrapolation share one sweep; --unfused makes it 4).  The
+slow step with the in-sweep norm, gate update.  By default that is 3 sweeps + 1 tiny
+kernel moving 72 bytes per parameter (--flow deferred: the first probe step leaves m, v
+to the fused second-probe + extrapolation sweep); --flow fused moves 84, --flow unfused
+(the four separate calls) 94.  The
 three gradient buffers are synthetic and already resident.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
@@ -30,8 +32,14 @@ if ROOT not in sys.path:
 METRIC = "GXPO active-step params/sec"
 UNIT = "params/s"
 BYTES_STEP_ADAMW = 26      # R theta, m, v (12) + g bf16 (2); W theta, m, v (12)
+BYTES_STEP_DEFERRED = 18   # R theta, m, v (12) + g0 (2); W theta1 (4): m, v stay as they are
 BYTES_EXTRAP = 16          # R theta2, theta0 (8) + g0, g1 bf16 (4); W theta-tilde (4)
 BYTES_FUSED = 32           # R theta1, theta0, m, v (16) + g0, g1 (4); W theta-tilde, m, v (12)
+BYTES_FUSED_DEFERRED = 28  # R theta0, m, v (12) + g0, g1 (4); W theta-tilde, m, v (12)
+# which kernel function serves which call
+KERNEL_OF = {"probe_step0": "step_kernel", "probe_step0_deferred": "step_kernel", "probe_step1": "step_kernel",
+             "slow_step": "step_kernel", "fallback_step": "step_kernel", "extrapolate": "extrap_kernel",
+             "probe_extrapolate": "fused_kernel", "probe_extrapolate_deferred": "fused_kernel"}
 
 
 def parse_args():
@@ -52,8 +60,9 @@ def parse_args():
     ap.add_argument("--ctas", type=int, default=0)
     ap.add_argument("--unit-tiles", type=int, default=0)
     ap.add_argument("--fallback", action="store_true", help="time the single-pass fallback step")
-    ap.add_argument("--unfused", action="store_true",
-                    help="probe step 1 and extrapolate as two sweeps (94 B/param) instead of one (84)")
+    ap.add_argument("--flow", default="deferred", choices=["deferred", "fused", "unfused"],
+                    help="deferred: probe_step_deferred + probe_extrapolate (72 B/param, default); "
+                         "fused: probe_step(0) + probe_extrapolate (84); unfused: the four separate sweeps (94)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-params", type=int, default=1 << 26)
@@ -83,22 +92,27 @@ def measured_peak_gbs():
         return 6650.0, "fallback"
 
 
-def recorded_traffic_per_param():
-    """DRAM bytes per parameter of the dominant kernel, from the committed ncu summary.
-    The summary records the hash of the kernel source it was taken from; once that
-    source has changed the counters no longer describe the kernel and None is returned."""
+def recorded_traffic_per_param(kernel_fn, calls):
+    """DRAM bytes per parameter of `kernel_fn`, averaged over the named calls, from the
+    committed ncu summary profiles/<kernel_fn>_adamw_bf16_flat134m.txt (lines
+    "dram_bytes_per_param[<call>]: X").  The summary records the hash of the kernel source
+    it was taken from; once that source has changed the counters no longer describe the
+    kernel and None is returned."""
     import hashlib
     import re
-    summary = os.path.join(ROOT, "profiles", "step_kernel_adamw_bf16_flat134m.txt")
+    summary = os.path.join(ROOT, "profiles", f"{kernel_fn}_adamw_bf16_flat134m.txt")
     source = os.path.join(ROOT, "paper_2605_06755_b200", "csrc", "gxpo_kernels.cuh")
     try:
         text = open(summary).read()
         want = re.search(r"^kernel_source_sha256:\s*([0-9a-f]{64})", text, re.M).group(1)
-        per_param = float(re.search(r"^dram_bytes_per_param:\s*([0-9.]+)", text, re.M).group(1))
         have = hashlib.sha256(open(source, "rb").read()).hexdigest()
+        if have != want:
+            return None
+        vals = [float(re.search(r"^dram_bytes_per_param\[%s\]:\s*([0-9.]+)" % re.escape(c), text, re.M).group(1))
+                for c in calls]
+        return statistics.mean(vals)
     except Exception:
         return None
-    return per_param if have == want else None
 
 
 # ----------------------------------------------------------------------------
@@ -283,9 +297,10 @@ def run_ours(args):
     if world > 1:
         ctx.set_sumsq_buffer(sumsq.data_ptr())
 
-    fused = not args.unfused
-    names = ["probe_step0", "probe_extrapolate", "slow_step"] if fused else \
-        ["probe_step0", "probe_step1", "extrapolate", "slow_step"]
+    flow = args.flow
+    names = {"deferred": ["probe_step0_deferred", "probe_extrapolate_deferred", "slow_step"],
+             "fused": ["probe_step0", "probe_extrapolate", "slow_step"],
+             "unfused": ["probe_step0", "probe_step1", "extrapolate", "slow_step"]}[flow]
     if args.fallback:
         names = ["fallback_step"]
     n_ev = len(names) + 1
@@ -299,9 +314,12 @@ def run_ours(args):
             ctx.probe_step(-1, stream)
             mark(1)
             return None
-        ctx.probe_step(0, stream)
+        if flow == "deferred":
+            ctx.probe_step_deferred(stream)
+        else:
+            ctx.probe_step(0, stream)
         mark(1)
-        if fused:
+        if flow != "unfused":
             ctx.probe_extrapolate(stream)
             mark(2)
         else:
@@ -351,23 +369,29 @@ def run_ours(args):
     per = {nm: statistics.mean(evs[s][i].elapsed_time(evs[s][i + 1]) for s in range(args.steps))
            for i, nm in enumerate(names)}
     peak, peak_kind = measured_peak_gbs()
-    alg_bytes = {"probe_step0": BYTES_STEP_ADAMW + (4 if args.placement == 1 else 0),
+    snap = 4 if args.placement == 1 else 0          # SNAPSHOT placement: probe 0 also copies theta^t
+    alg_bytes = {"probe_step0": BYTES_STEP_ADAMW + snap, "probe_step0_deferred": BYTES_STEP_DEFERRED + snap,
                  "probe_step1": BYTES_STEP_ADAMW, "extrapolate": BYTES_EXTRAP,
-                 "probe_extrapolate": BYTES_FUSED, "slow_step": BYTES_STEP_ADAMW,
-                 "fallback_step": BYTES_STEP_ADAMW}
-    kernels = {nm: {"ms": ms, "bytes_per_param": alg_bytes[nm],
+                 "probe_extrapolate": BYTES_FUSED, "probe_extrapolate_deferred": BYTES_FUSED_DEFERRED,
+                 "slow_step": BYTES_STEP_ADAMW, "fallback_step": BYTES_STEP_ADAMW}
+    kernels = {nm: {"kernel": KERNEL_OF[nm], "ms": ms, "bytes_per_param": alg_bytes[nm],
                     "gbs": alg_bytes[nm] * d / (ms * 1e-3) / 1e9} for nm, ms in per.items()}
-    # dominant kernel: the AdamW sweep (step_kernel), launched for probe step 0 (PINGPONG
-    # placement: plain 26 B/param), the slow step and the fallback step
-    dom = [nm for nm in ("probe_step0", "probe_step1", "slow_step", "fallback_step")
-           if nm in per and alg_bytes[nm] == BYTES_STEP_ADAMW]
-    step_ms = statistics.mean(per[nm] for nm in dom)
-    achieved = BYTES_STEP_ADAMW * d / (step_ms * 1e-3) / 1e9
-    tpp = recorded_traffic_per_param()
-    roofline = {"bound": "hbm", "kernel": "step_kernel (AdamW sweep: probe step, slow step, fallback step)",
-                "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "peak_kind": f"of {peak_kind}", "traffic": (tpp * d if tpp else None),
-                "algorithmic_bytes_per_launch": BYTES_STEP_ADAMW * d, "launches_averaged": dom}
+    # dominant kernel = the kernel function with the largest share of the step; its figures
+    # are averages over its launches in one step (algorithmic bytes and duration alike)
+    by_fn = {}
+    for nm, ms in per.items():
+        by_fn.setdefault(KERNEL_OF[nm], []).append(nm)
+    dom_fn = max(by_fn, key=lambda f: sum(per[nm] for nm in by_fn[f]))
+    dom = by_fn[dom_fn]
+    dom_bytes = statistics.mean(alg_bytes[nm] for nm in dom) * d
+    dom_ms = statistics.mean(per[nm] for nm in dom)
+    achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
+    tpp = recorded_traffic_per_param(dom_fn, dom)
+    roofline = {"bound": "hbm", "kernel": dom_fn, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                "traffic": (tpp * d if tpp else None),
+                "algorithmic_bytes_per_launch": dom_bytes, "ms_per_launch": dom_ms,
+                "launches_averaged": dom, "share_of_step": sum(per[nm] for nm in dom) / sum(per.values())}
     step_bytes = sum(alg_bytes[nm] for nm in names) * d
     whole_gbs = step_bytes / (ms_step * 1e-3) / 1e9
 
@@ -380,8 +404,9 @@ def run_ours(args):
                    "K": args.K, "alpha": args.alpha, "lr": args.lr, "grad_dtype": "bf16",
                    "placement": ["pingpong", "snapshot"][args.placement],
                    "step": "fallback (single pass)" if args.fallback else
-                   ("active (probe, fused probe+extrapolate, slow step, gate)" if fused else
-                    "active (probe, probe, extrapolate, slow step, gate)"),
+                   {"deferred": "active (probe with deferred state, probe+extrapolate in one sweep, slow step, gate)",
+                    "fused": "active (probe, probe+extrapolate in one sweep, slow step, gate)",
+                    "unfused": "active (probe, probe, extrapolate, slow step, gate)"}[flow],
                    "g_slow_aliases_g0": alias, "l2": "inputs larger than L2 (no flush needed)",
                    "parallelism": f"dp{world} (independent shards, one 8-byte all-reduce per step)" if world > 1 else "1 GPU"},
         "hbm_gbs_whole_step": whole_gbs, "hbm_frac_whole_step": whole_gbs / peak,

@@ -159,8 +159,21 @@ gxpo_status gxpo_extrapolate(gxpo_ctx* ctx, void* stream);
 /* gxpo_probe_step(ctx, 1) and gxpo_extrapolate in ONE sweep: Algorithm 1 takes no
  * backward pass at theta^{t,2}, so that point never has to reach memory.  Same
  * per-coordinate arithmetic, bit-identical theta-tilde, m and v; 32 instead of
- * 26 + 16 bytes per parameter.  state: PROBED0 -> EXTRAPOLATED. */
+ * 26 + 16 bytes per parameter.  state: PROBED0 (or PROBED0_DEFERRED, see
+ * gxpo_probe_step_deferred) -> EXTRAPOLATED. */
 gxpo_status gxpo_probe_extrapolate(gxpo_ctx* ctx, void* stream);
+
+/* The first fast step for callers that will take the second one with
+ * gxpo_probe_extrapolate: theta^{t,1} is written exactly as by gxpo_probe_step(ctx, 0)
+ * (the caller's second backward pass needs it), but m and v are NOT written; they stay
+ * at their start-of-step values until gxpo_probe_extrapolate replays this step in
+ * registers (same function, same bits, hence the same theta^{t,1}), takes the second
+ * step and writes m and v once.  Results are bit-identical to the other call sequences;
+ * the active step moves 18 + 28 + 26 = 72 instead of 26 + 32 + 26 = 84 bytes per
+ * parameter.  The optimizer step count advances as usual.  Until gxpo_probe_extrapolate
+ * has run, m and v in memory are one step behind and g0 must stay intact.
+ * state: IDLE -> PROBED0_DEFERRED; from there only gxpo_probe_extrapolate is legal. */
+gxpo_status gxpo_probe_step_deferred(gxpo_ctx* ctx, void* stream);
 
 /* Algorithm 1, "slow correction": theta^{t+1} <- OptimStep(theta-tilde, g_slow), in
  * place in `theta`, and sum(g_slow^2) accumulated in the same sweep (float64,

@@ -62,6 +62,7 @@ _sigs = {
     "gxpo_destroy": (None, [_vp]),
     "gxpo_bind": (ctypes.c_int, [_vp, ctypes.POINTER(Tensor), ctypes.c_int]),
     "gxpo_probe_step": (ctypes.c_int, [_vp, ctypes.c_int, _vp]),
+    "gxpo_probe_step_deferred": (ctypes.c_int, [_vp, _vp]),
     "gxpo_extrapolate": (ctypes.c_int, [_vp, _vp]),
     "gxpo_probe_extrapolate": (ctypes.c_int, [_vp, _vp]),
     "gxpo_slow_step": (ctypes.c_int, [_vp, _vp]),
@@ -187,6 +188,9 @@ class Context:
     def probe_step(self, which: int, stream=None):
         self._check(_lib.gxpo_probe_step(self._h, which, _stream_ptr(stream)))
 
+    def probe_step_deferred(self, stream=None):
+        self._check(_lib.gxpo_probe_step_deferred(self._h, _stream_ptr(stream)))
+
     def extrapolate(self, stream=None):
         self._check(_lib.gxpo_extrapolate(self._h, _stream_ptr(stream)))
 
@@ -247,11 +251,16 @@ class Context:
 
     # -- convenience: the calls of one active step in Algorithm 1's order, for callers
     #    whose three gradient buffers are already filled (benchmarks, replay) --------
-    def active_step(self, stream=None, allow_nonfinite: bool = False, fused: bool = False) -> GateResult:
-        self.probe_step(0, stream)
-        if fused:
+    def active_step(self, stream=None, allow_nonfinite: bool = False, fused: bool = False,
+                    deferred: bool = False) -> GateResult:
+        if deferred:
+            self.probe_step_deferred(stream)
+            self.probe_extrapolate(stream)
+        elif fused:
+            self.probe_step(0, stream)
             self.probe_extrapolate(stream)
         else:
+            self.probe_step(0, stream)
             self.probe_step(1, stream)
             self.extrapolate(stream)
         self.slow_step(stream)

@@ -17,10 +17,11 @@ namespace {
 
 constexpr int kDefaultUnitShift = 0;   // whole chunks
 constexpr int kDefaultCtasStep = 2;    // measured best for the 14R/12W sweep
+constexpr int kDefaultCtasStepLight = 3;  // 14R/4W (deferred first probe): read-heavy, wants more loads in flight
 constexpr int kDefaultCtasExtrap = 4;  // the extrapolation needs more warps to cover its arithmetic
 constexpr int kDefaultCtasFused = 3;
 
-enum Phase { IDLE = 0, PROBED0 = 1, PROBED1 = 2, EXTRAPOLATED = 3, SLOW_DONE = 4 };
+enum Phase { IDLE = 0, PROBED0 = 1, PROBED1 = 2, EXTRAPOLATED = 3, SLOW_DONE = 4, PROBED0_DEFERRED = 5 };
 
 struct Staging {                       // device pieces for gxpo_step_host
     long long elems = 0;
@@ -148,6 +149,7 @@ StepParams make_step_params(gxpo_ctx* c, int which_grad, int in_sel, int out_sel
     p.out_sel = out_sel;
     p.snapshot = snapshot;
     p.want_norm = want_norm;
+    p.write_state = 1;
     const gxpo_opt_cfg& o = c->opt;
     p.lr = (float)o.lr;
     if (o.kind == GXPO_OPT_ADAMW) {
@@ -183,13 +185,17 @@ ExtrapFn pick_extrap(bool bf16, int variant) {
     if (variant == 1) return bf16 ? extrap_kernel<uint16_t, 4> : extrap_kernel<float, 4>;
     return bf16 ? extrap_kernel<uint16_t, 8> : extrap_kernel<float, 8>;
 }
-FusedFn pick_fused(bool adamw, bool bf16, int variant) {
+template <bool DEFER>
+FusedFn pick_fused_t(bool adamw, bool bf16, int variant) {
     if (variant == 1) {
-        if (adamw) return bf16 ? fused_kernel<true, uint16_t, 4> : fused_kernel<true, float, 4>;
-        return bf16 ? fused_kernel<false, uint16_t, 4> : fused_kernel<false, float, 4>;
+        if (adamw) return bf16 ? fused_kernel<true, uint16_t, 4, DEFER> : fused_kernel<true, float, 4, DEFER>;
+        return bf16 ? fused_kernel<false, uint16_t, 4, DEFER> : fused_kernel<false, float, 4, DEFER>;
     }
-    if (adamw) return bf16 ? fused_kernel<true, uint16_t, 8> : fused_kernel<true, float, 8>;
-    return bf16 ? fused_kernel<false, uint16_t, 8> : fused_kernel<false, float, 8>;
+    if (adamw) return bf16 ? fused_kernel<true, uint16_t, 8, DEFER> : fused_kernel<true, float, 8, DEFER>;
+    return bf16 ? fused_kernel<false, uint16_t, 8, DEFER> : fused_kernel<false, float, 8, DEFER>;
+}
+FusedFn pick_fused(bool adamw, bool bf16, int variant, bool defer) {
+    return defer ? pick_fused_t<true>(adamw, bf16, variant) : pick_fused_t<false>(adamw, bf16, variant);
 }
 
 // Launch one OptimStep sweep over either the bound list (chunks != null) or one
@@ -203,7 +209,8 @@ gxpo_status launch_step(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, co
     }
     const bool adamw = c->opt.kind == GXPO_OPT_ADAMW;
     StepFn fn = pick_step(adamw, c->grad_dtype == GXPO_BF16, c->variant);
-    const int grid = grid_for(c, (const void*)fn, num_chunks << c->unit_shift, kDefaultCtasStep);
+    const int grid = grid_for(c, (const void*)fn, num_chunks << c->unit_shift,
+                              (adamw && !p.write_state) ? kDefaultCtasStepLight : kDefaultCtasStep);
     fn<<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, c->unit_shift, c->d_partials, c->d_ticket, sumsq);
     c->launches += 1;
     CUDA_TRY(c, cudaGetLastError());
@@ -222,9 +229,9 @@ gxpo_status launch_extrap(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, 
 }
 
 gxpo_status launch_fused(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
-                         long long num_chunks, const TensorDesc& flat, const FusedParams& p) {
+                         long long num_chunks, const TensorDesc& flat, const FusedParams& p, bool defer) {
     if (num_chunks <= 0) return GXPO_OK;
-    FusedFn fn = pick_fused(c->opt.kind == GXPO_OPT_ADAMW, c->grad_dtype == GXPO_BF16, c->variant);
+    FusedFn fn = pick_fused(c->opt.kind == GXPO_OPT_ADAMW, c->grad_dtype == GXPO_BF16, c->variant, defer);
     const int grid = grid_for(c, (const void*)fn, num_chunks << c->unit_shift, kDefaultCtasFused);
     fn<<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, c->unit_shift);
     c->launches += 1;
@@ -475,6 +482,8 @@ gxpo_status gxpo_probe_step(gxpo_ctx* c, int which, void* stream) {
         c->phase = PROBED0;
         return GXPO_OK;
     }
+    if (c->phase == PROBED0_DEFERRED)
+        return fail(c, GXPO_ERR_STATE, "after gxpo_probe_step_deferred only gxpo_probe_extrapolate can take the second probe step");
     if (c->phase != PROBED0) return fail(c, GXPO_ERR_STATE, "probe step 1 must follow probe step 0");
     c->t_opt += 1;
     StepParams p = (place == GXPO_PLACE_PINGPONG) ? make_step_params(c, 1, 1, 1, 0, 0)
@@ -482,6 +491,22 @@ gxpo_status gxpo_probe_step(gxpo_ctx* c, int which, void* stream) {
     gxpo_status st = launch_step(c, s, c->d_descs, c->d_chunks, c->num_chunks, none, p, c->d_sumsq);
     if (st != GXPO_OK) { c->t_opt -= 1; return st; }
     c->phase = PROBED1;
+    return GXPO_OK;
+}
+
+gxpo_status gxpo_probe_step_deferred(gxpo_ctx* c, void* stream) {
+    if (!c) return GXPO_ERR_INVALID_ARG;
+    if (!c->bound) return fail(c, GXPO_ERR_STATE, "nothing bound: call gxpo_bind first");
+    if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "probe step 0 must start a step");
+    if (!gate_active(c)) return fail(c, GXPO_ERR_STATE, "gate has tripped (s*=%lld, t=%lld): only fallback steps are legal", c->s_star, c->t);
+    const TensorDesc none = {};
+    c->t_opt += 1;
+    StepParams p = (c->cfg.placement == GXPO_PLACE_PINGPONG) ? make_step_params(c, 0, 0, 1, 0, 0)
+                                                             : make_step_params(c, 0, 0, 0, 1, 0);
+    p.write_state = 0;
+    gxpo_status st = launch_step(c, (cudaStream_t)stream, c->d_descs, c->d_chunks, c->num_chunks, none, p, c->d_sumsq);
+    if (st != GXPO_OK) { c->t_opt -= 1; return st; }
+    c->phase = PROBED0_DEFERRED;
     return GXPO_OK;
 }
 
@@ -498,14 +523,17 @@ gxpo_status gxpo_extrapolate(gxpo_ctx* c, void* stream) {
 
 gxpo_status gxpo_probe_extrapolate(gxpo_ctx* c, void* stream) {
     if (!c) return GXPO_ERR_INVALID_ARG;
-    if (c->phase != PROBED0) return fail(c, GXPO_ERR_STATE, "fused probe+extrapolate must follow probe step 0");
+    if (c->phase != PROBED0 && c->phase != PROBED0_DEFERRED)
+        return fail(c, GXPO_ERR_STATE, "fused probe+extrapolate must follow probe step 0");
     const TensorDesc none = {};
     const int place = c->cfg.placement;
-    c->t_opt += 1;
+    const bool defer = c->phase == PROBED0_DEFERRED;
     FusedParams p;
+    p.step0 = make_step_params(c, 0, 0, 0, 0, 0);       // constants of the first probe step (replayed when deferred)
+    c->t_opt += 1;
     p.step = (place == GXPO_PLACE_PINGPONG) ? make_step_params(c, 1, 1, 1, 0, 0) : make_step_params(c, 1, 0, 0, 0, 0);
     p.ex = make_extrap_params(c, place);
-    gxpo_status st = launch_fused(c, (cudaStream_t)stream, c->d_descs, c->d_chunks, c->num_chunks, none, p);
+    gxpo_status st = launch_fused(c, (cudaStream_t)stream, c->d_descs, c->d_chunks, c->num_chunks, none, p, defer);
     if (st != GXPO_OK) { c->t_opt -= 1; return st; }
     c->phase = EXTRAPOLATED;
     return GXPO_OK;
@@ -693,9 +721,10 @@ gxpo_status gxpo_step_host(gxpo_ctx* c, const gxpo_tensor* list, int count, long
                 if (rs != GXPO_OK) return rs;
                 c->t_opt = t_opt0 + 2;
                 FusedParams fp;
+                fp.step0 = make_step_params(c, 0, 0, 0, 0, 0);
                 fp.step = make_step_params(c, 1, 1, 1, 0, 0);
                 fp.ex = make_extrap_params(c, GXPO_PLACE_PINGPONG);
-                rs = launch_fused(c, s, nullptr, nullptr, nch, d, fp);
+                rs = launch_fused(c, s, nullptr, nullptr, nch, d, fp, false);
                 if (rs != GXPO_OK) return rs;
                 c->t_opt = t_opt0 + 3;
                 rs = launch_step(c, s, nullptr, nullptr, nch, d, make_step_params(c, 2, 0, 0, 0, 1), st.piece_sumsq + 1);
@@ -917,6 +946,7 @@ extern "C" gxpo_status gxpo_slow_step_noalloc(float* theta, float* m, float* v, 
     std::memset(&p, 0, sizeof(p));
     p.which_grad = 2;
     p.want_norm = 1;
+    p.write_state = 1;
     p.lr = (float)opt->lr;
     if (adamw) {
         const double t = (double)t_opt, b1 = opt->beta1, b2 = opt->beta2, lr = opt->lr;

@@ -321,6 +321,70 @@ def test_fused_probe_extrapolate_is_bit_identical_to_the_two_calls(kind, grad_dt
     assert (outs[0][6], outs[1][6]) == (5, 4)
 
 
+@pytest.mark.parametrize("kind,grad_dtype", [("adamw", "bf16"), ("adamw", "f32"), ("gd", "f32"), ("gd", "bf16")])
+@pytest.mark.parametrize("placement", [0, 1])
+def test_deferred_state_flow_is_bit_identical_to_the_four_calls(kind, grad_dtype, placement):
+    """gxpo_probe_step_deferred leaves m, v alone and gxpo_probe_extrapolate replays the
+    first probe step in registers: theta^{t,1}, theta-tilde, the final theta, m, v and the
+    norm must equal, bit for bit, what probe 0, probe 1, extrapolate give -- the sequence
+    the other tests compare with the oracle -- over two consecutive steps."""
+    b = _binding()
+    sizes = [3 * 32768 + 5, 2047, 1, 40003, 4096]
+    offsets = [0, 0, 0, 1, 0]
+    outs = []
+    for deferred in (False, True):
+        probs = [_problem(n, seed=80 + i, grad_dtype=grad_dtype, zero_frac=0.03, offset=off)
+                 for i, (n, off) in enumerate(zip(sizes, offsets))]
+        ctx, cfg, opt = _ctx(b, grad_dtype, kind=b.OPT_ADAMW if kind == "adamw" else b.OPT_GD, lr=1e-3,
+                             K=5, alpha=0.5, placement=placement)
+        ctx.bind([p.ptrs() for p in probs])
+        rec = []
+        for step in range(2):
+            m_before = [gu.to_host_f64(p.m) for p in probs]
+            if deferred:
+                ctx.probe_step_deferred()
+                for p, mb in zip(probs, m_before):          # optimizer state not written yet
+                    np.testing.assert_array_equal(gu.to_host_f64(p.m), mb)
+                rec.append([gu.to_host_f64(p.work if placement == 0 else p.theta) for p in probs])
+                ctx.probe_extrapolate()
+            else:
+                ctx.probe_step(0)
+                rec.append([gu.to_host_f64(p.work if placement == 0 else p.theta) for p in probs])
+                ctx.probe_step(1)
+                ctx.extrapolate()
+            rec.append([gu.to_host_f64(p.theta) for p in probs])
+            ctx.slow_step()
+            res = ctx.gate_update(allow_nonfinite=True)
+            rec.append([gu.to_host_f64(p.theta) for p in probs])
+            rec.append([gu.to_host_f64(p.m) for p in probs])
+            rec.append([gu.to_host_f64(p.v) for p in probs])
+            rec.append([np.array(res.norm)])
+        outs.append((rec, ctx.optimizer_steps(), ctx.launch_count()))
+        ctx.close()
+    for a, c in zip(outs[0][0], outs[1][0]):
+        for x, y in zip(a, c):
+            np.testing.assert_array_equal(x, y)
+    assert outs[0][1] == outs[1][1] == 6
+    assert (outs[0][2], outs[1][2]) == (10, 8)
+
+
+def test_deferred_call_order():
+    b = _binding()
+    pr = _problem(1000, 1, "bf16")
+    ctx, cfg, opt = _ctx(b, "bf16")
+    ctx.bind([pr.ptrs()])
+    ctx.probe_step_deferred()
+    for call in (lambda: ctx.probe_step(1), ctx.extrapolate, ctx.slow_step, ctx.gate_update,
+                 ctx.probe_step_deferred, lambda: ctx.probe_step(0), lambda: ctx.probe_step(-1)):
+        with pytest.raises(b.GxpoError) as e:
+            call()
+        assert e.value.status == b.ERR_STATE
+    ctx.probe_extrapolate()
+    ctx.slow_step()
+    assert ctx.gate_update().t == 1 and ctx.optimizer_steps() == 3
+    ctx.close()
+
+
 def test_fused_call_order():
     b = _binding()
     pr = _problem(1000, 1, "bf16")
