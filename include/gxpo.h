@@ -227,8 +227,8 @@ gxpo_status gxpo_step_host(gxpo_ctx* ctx, const gxpo_tensor* list, int count,
 
 /* Launch-shape knobs, for benchmarking: resident CTAs per SM (0 = default), the
  * memory-access variant (0 = default, 1 = 128-bit loads, 2 = 256-bit loads) and the
- * number of 2048-element tiles a CTA takes per round-robin turn (0 = default; 1, 2,
- * 4, 8 or 16).  Element-wise results are identical across all settings; only the
+ * number of 2048-element tiles a CTA takes per round-robin turn (0 = default: 16, or
+ * 8 / 4 for lists of only a few thousand 32768-element chunks; else 1, 2, 4, 8 or 16).  Element-wise results are identical across all settings; only the
  * summation order of the norm changes. */
 gxpo_status gxpo_tune(gxpo_ctx* ctx, int ctas_per_sm, int variant, int unit_tiles);
 

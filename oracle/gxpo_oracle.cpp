@@ -23,6 +23,8 @@
  *   l2norm                      : closed forms, a library norm
  *   gate                        : hand-built norm streams, a library mean/std,
  *                                 printed (shutoff step, total backward passes) rows
+ *   active-step diagnostics     : a hand-computed example, closed forms on the diagonal
+ *                                 quadratic, library mean/std/dot, degenerate cases
  * The AdamW *hyper-parameter defaults* and the gate's window, epsilon, warm-up
  * and std convention are not fixed by the paper: for those, parity is unpinned
  * (they are parameters here, never constants).
@@ -130,6 +132,79 @@ double gxo_sum_squares(const double* g, int64_t n) {
 }
 
 double gxo_l2norm(const double* g, int64_t n) { return std::sqrt(gxo_sum_squares(g, n)); }
+
+/* ---- Per-step diagnostics of the active phase, the quantities the paper's appendix
+ *      tabulates ("Active-phase GXPO diagnostics": gradient norms, cos(g0, g_slow),
+ *      retention ratio mean +- std, ||Delta_K|| / ||Delta_2||, scale mean, inactive
+ *      fraction).  Plain definitions, two passes where a mean is needed first.
+ *
+ *      A coordinate is "regular" unless it is active and its ratio r or its scale
+ *      factor does not fit a finite float (the update stores float32, so such a
+ *      coordinate has no usable scale); irregular coordinates are counted and left out
+ *      of the ratio, scale and displacement statistics.  Inactive coordinates have
+ *      scale 1 and no ratio.
+ *        out[0..2]  ||g0||, ||g1||, ||g_slow||           (all coordinates)
+ *        out[3]     cos(g0, g_slow) = <g0, g_slow> / (||g0|| ||g_slow||)
+ *        out[4..5]  mean and population std of r over regular active coordinates
+ *        out[6]     mean of scale over regular coordinates (inactive ones count as 1)
+ *        out[7]     ||Delta_K|| / ||Delta_2||, Delta_2 = theta2 - theta0,
+ *                   Delta_K = Delta_2 * scale, over regular coordinates
+ *        out[8]     inactive fraction = 1 - |A_t| / n
+ *        out[9]     |A_t|;   out[10]  number of irregular coordinates              */
+void gxo_active_diagnostics(const double* theta0, const double* theta2, const double* g0,
+                            const double* g1, const double* g_slow, int64_t n, int K, double delta,
+                            double den_eps, double* out) {
+    double s00 = 0.0, s11 = 0.0, sss = 0.0, s0s = 0.0;
+    double sum_r = 0.0, sum_scale = 0.0, d2 = 0.0, dk = 0.0;
+    int64_t n_active = 0, n_irregular = 0, n_ratio = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        s00 += g0[i] * g0[i];
+        s11 += g1[i] * g1[i];
+        sss += g_slow[i] * g_slow[i];
+        s0s += g0[i] * g_slow[i];
+        double scale = 1.0;
+        if (std::fabs(g0[i]) > delta) {
+            n_active += 1;
+            const double r = g1[i] / g0[i];
+            const double s2 = geom_sum(r, 2);
+            if (!(den_eps > 0.0 && std::fabs(s2) <= den_eps)) scale = geom_sum(r, K) / s2;
+            if (!std::isfinite(static_cast<float>(r)) || !std::isfinite(static_cast<float>(scale))) {
+                n_irregular += 1;
+                continue;
+            }
+            sum_r += r;
+            n_ratio += 1;
+        }
+        const double d = theta2[i] - theta0[i];
+        sum_scale += scale;
+        d2 += d * d;
+        dk += (d * scale) * (d * scale);
+    }
+    const double nan = std::numeric_limits<double>::quiet_NaN();
+    const double mean_r = n_ratio > 0 ? sum_r / n_ratio : nan;
+    double var_r = 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+        if (!(std::fabs(g0[i]) > delta)) continue;
+        const double r = g1[i] / g0[i];
+        double scale = 1.0;
+        const double s2 = geom_sum(r, 2);
+        if (!(den_eps > 0.0 && std::fabs(s2) <= den_eps)) scale = geom_sum(r, K) / s2;
+        if (!std::isfinite(static_cast<float>(r)) || !std::isfinite(static_cast<float>(scale))) continue;
+        var_r += (r - mean_r) * (r - mean_r);
+    }
+    const int64_t n_regular = n - n_irregular;
+    out[0] = std::sqrt(s00);
+    out[1] = std::sqrt(s11);
+    out[2] = std::sqrt(sss);
+    out[3] = s0s / (std::sqrt(s00) * std::sqrt(sss));
+    out[4] = mean_r;
+    out[5] = n_ratio > 0 ? std::sqrt(var_r / n_ratio) : nan;
+    out[6] = n_regular > 0 ? sum_scale / n_regular : nan;
+    out[7] = std::sqrt(dk) / std::sqrt(d2);
+    out[8] = n > 0 ? 1.0 - static_cast<double>(n_active) / n : nan;
+    out[9] = static_cast<double>(n_active);
+    out[10] = static_cast<double>(n_irregular);
+}
 
 /* ---- Rolling z-score gate ("Adaptive rule in practice"; Algorithm 1, the block
  *      after the slow correction).

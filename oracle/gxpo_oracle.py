@@ -54,6 +54,9 @@ def lib():
         L.gxo_sum_squares.restype = ctypes.c_double
         L.gxo_l2norm.argtypes = [_f64p, _i64]
         L.gxo_l2norm.restype = ctypes.c_double
+        L.gxo_active_diagnostics.argtypes = [_f64p] * 5 + [_i64, ctypes.c_int, ctypes.c_double,
+                                             ctypes.c_double, _f64p]
+        L.gxo_active_diagnostics.restype = None
         L.gxo_gate_create.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.c_int,
                                       ctypes.c_int, ctypes.c_int]
         L.gxo_gate_create.restype = ctypes.c_void_p
@@ -142,6 +145,18 @@ def sum_squares(g) -> float:
 
 def l2norm(g) -> float:
     return float(lib().gxo_l2norm(_p(g), g.size))
+
+
+DIAG_FIELDS = ("g0_norm", "g1_norm", "gslow_norm", "cos_g0_gslow", "ratio_mean", "ratio_std",
+               "scale_mean", "disp_ratio", "inactive_frac", "n_active", "n_irregular")
+
+
+def active_diagnostics(theta0, theta2, g0, g1, g_slow, K, delta, den_eps=0.0) -> dict:
+    """The appendix's active-phase diagnostics for one step (see the C++ header comment)."""
+    out = np.empty(len(DIAG_FIELDS), dtype=np.float64)
+    lib().gxo_active_diagnostics(_p(theta0), _p(theta2), _p(g0), _p(g1), _p(g_slow), theta0.size,
+                                 int(K), float(delta), float(den_eps), _p(out))
+    return dict(zip(DIAG_FIELDS, out.tolist()))
 
 
 def backward_budget(s_star: int, T: int) -> int:

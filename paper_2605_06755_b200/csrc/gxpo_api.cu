@@ -15,7 +15,6 @@ using namespace gxpo;
 
 namespace {
 
-constexpr int kDefaultUnitShift = 0;   // whole chunks
 constexpr int kDefaultCtasStep = 2;    // measured best for the 14R/12W sweep
 constexpr int kDefaultCtasStepLight = 3;  // 14R/4W (deferred first probe): read-heavy, wants more loads in flight
 constexpr int kDefaultCtasExtrap = 4;  // the extrapolation needs more warps to cover its arithmetic
@@ -46,7 +45,7 @@ struct gxpo_ctx {
     int sm_count;
     int ctas_per_sm;                   // 0 = default
     int variant;                       // 1 = 128-bit, 2 = 256-bit
-    int unit_shift;                    // work unit = kChunk >> unit_shift elements
+    int unit_shift;                    // work unit = kChunk >> unit_shift elements; -1 = choose per launch
     Phase phase;
     // bound list
     TensorDesc* d_descs;
@@ -140,6 +139,18 @@ int grid_for(gxpo_ctx* c, const void* kernel, long long units, int default_per_s
     return (int)g;
 }
 
+// Work unit for one launch.  Whole chunks (16 tiles) have the least per-unit overhead
+// and are right for lists of billions of parameters; a list of only a few thousand
+// chunks is dealt in quarter or half chunks so that every CTA still gets tens of units
+// and the last wave is short.
+int unit_shift_for(const gxpo_ctx* c, long long num_chunks) {
+    if (c->unit_shift >= 0) return c->unit_shift;
+    const long long want = 32LL * c->sm_count * kDefaultCtasStep;
+    int sh = 0;
+    while (sh < 2 && (num_chunks << sh) < want) ++sh;
+    return sh;
+}
+
 StepParams make_step_params(gxpo_ctx* c, int which_grad, int in_sel, int out_sel, int snapshot,
                             int want_norm) {
     StepParams p;
@@ -209,9 +220,10 @@ gxpo_status launch_step(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, co
     }
     const bool adamw = c->opt.kind == GXPO_OPT_ADAMW;
     StepFn fn = pick_step(adamw, c->grad_dtype == GXPO_BF16, c->variant);
-    const int grid = grid_for(c, (const void*)fn, num_chunks << c->unit_shift,
+    const int ush = unit_shift_for(c, num_chunks);
+    const int grid = grid_for(c, (const void*)fn, num_chunks << ush,
                               (adamw && !p.write_state) ? kDefaultCtasStepLight : kDefaultCtasStep);
-    fn<<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, c->unit_shift, c->d_partials, c->d_ticket, sumsq);
+    fn<<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, ush, c->d_partials, c->d_ticket, sumsq);
     c->launches += 1;
     CUDA_TRY(c, cudaGetLastError());
     return GXPO_OK;
@@ -221,8 +233,9 @@ gxpo_status launch_extrap(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, 
                           long long num_chunks, const TensorDesc& flat, const ExtrapParams& p) {
     if (num_chunks <= 0) return GXPO_OK;
     ExtrapFn fn = pick_extrap(c->grad_dtype == GXPO_BF16, c->variant);
-    const int grid = grid_for(c, (const void*)fn, num_chunks << c->unit_shift, kDefaultCtasExtrap);
-    fn<<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, c->unit_shift);
+    const int ush = unit_shift_for(c, num_chunks);
+    const int grid = grid_for(c, (const void*)fn, num_chunks << ush, kDefaultCtasExtrap);
+    fn<<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, ush);
     c->launches += 1;
     CUDA_TRY(c, cudaGetLastError());
     return GXPO_OK;
@@ -232,8 +245,9 @@ gxpo_status launch_fused(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, c
                          long long num_chunks, const TensorDesc& flat, const FusedParams& p, bool defer) {
     if (num_chunks <= 0) return GXPO_OK;
     FusedFn fn = pick_fused(c->opt.kind == GXPO_OPT_ADAMW, c->grad_dtype == GXPO_BF16, c->variant, defer);
-    const int grid = grid_for(c, (const void*)fn, num_chunks << c->unit_shift, kDefaultCtasFused);
-    fn<<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, c->unit_shift);
+    const int ush = unit_shift_for(c, num_chunks);
+    const int grid = grid_for(c, (const void*)fn, num_chunks << ush, kDefaultCtasFused);
+    fn<<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, ush);
     c->launches += 1;
     CUDA_TRY(c, cudaGetLastError());
     return GXPO_OK;
@@ -356,7 +370,7 @@ gxpo_status gxpo_create(const gxpo_cfg* cfg, const gxpo_opt_cfg* opt, int grad_d
     c->opt = *opt;
     c->grad_dtype = grad_dtype;
     c->variant = 2;
-    c->unit_shift = kDefaultUnitShift;
+    c->unit_shift = -1;
     c->s_star = -1;
     c->phase = IDLE;
     cudaError_t e = cudaGetDevice(&c->device);
@@ -605,12 +619,13 @@ gxpo_status gxpo_tune(gxpo_ctx* c, int ctas_per_sm, int variant, int unit_tiles)
     if (ctas_per_sm < 0 || ctas_per_sm > 16) return fail(c, GXPO_ERR_INVALID_ARG, "ctas_per_sm must be in [0, 16]");
     if (variant < 0 || variant > 2) return fail(c, GXPO_ERR_INVALID_ARG, "variant must be 0, 1 or 2");
     int ush = -1;
-    if (unit_tiles == 0) ush = kDefaultUnitShift;
+    const bool auto_unit = unit_tiles == 0;
+    if (auto_unit) ush = 0;
     for (int k = 0; k <= 4; ++k) if (unit_tiles == (kTilesPerChunk >> k)) ush = k;
     if (ush < 0) return fail(c, GXPO_ERR_INVALID_ARG, "unit_tiles must be 0, 1, 2, 4, 8 or 16");
     c->ctas_per_sm = ctas_per_sm;
     c->variant = variant == 0 ? 2 : variant;
-    c->unit_shift = ush;
+    c->unit_shift = auto_unit ? -1 : ush;
     return GXPO_OK;
 }
 

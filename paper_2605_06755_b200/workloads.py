@@ -65,6 +65,21 @@ def llama31_8b_shapes(layers: int = 32) -> List[Tuple[str, int]]:
     return decoder_shapes(layers, 4096, 14336, 32, 8, 128, 128256, qkv_bias=False)
 
 
+def lora_qwen25_7b_shapes(rank: int = 128, layers: int = 28) -> List[Tuple[str, int]]:
+    """Rank-`rank` LoRA adapters on the q, k, v, o projections of a Qwen2.5-7B-shaped
+    decoder (the paper's 7B setting): per layer four A matrices [rank x in] and four B
+    matrices [out x rank].  rank 128 -> 224 tensors of 65,536 or 458,752 elements,
+    80,740,352 parameters."""
+    hidden, q_out, kv_out = 3584, 28 * 128, 4 * 128
+    out: List[Tuple[str, int]] = []
+    for l in range(layers):
+        for name, fan_in, fan_out in (("q_proj", hidden, q_out), ("k_proj", hidden, kv_out),
+                                      ("v_proj", hidden, kv_out), ("o_proj", q_out, hidden)):
+            out.append((f"layers.{l}.{name}.lora_A", rank * fan_in))
+            out.append((f"layers.{l}.{name}.lora_B", fan_out * rank))
+    return out
+
+
 FLAT_QWEN25_1P5B = 1_540_000_000   # "flat 1.54e9-param buffer"
 
 
