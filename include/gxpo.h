@@ -197,6 +197,39 @@ gxpo_status gxpo_gate_update(gxpo_ctx* ctx, void* stream, gxpo_gate_result* out)
  * same reduced value on every rank the gates flip together. */
 gxpo_status gxpo_set_sumsq_buffer(gxpo_ctx* ctx, double* sumsq_dev);
 
+/* Per-step diagnostics of the active phase: the quantities the paper's appendix
+ * tabulates ("Active-phase GXPO diagnostics").  Off by default.  When on, the sums are
+ * gathered inside the extrapolation sweep (gxpo_extrapolate or gxpo_probe_extrapolate) at
+ * no extra memory traffic; only <g0, g_slow> needs one more pass over the two gradient
+ * buffers after the slow step (+4 bytes per parameter for bfloat16 gradients), and is
+ * skipped (cos = NaN) when some tensor's g_slow shares g0's buffer.
+ *   g0_norm, g1_norm, gslow_norm : Euclidean norms over all coordinates
+ *   cos_g0_gslow                 : <g0, g_slow> / (||g0|| ||g_slow||)
+ *   ratio_mean, ratio_std        : mean and population standard deviation of the
+ *                                  retention ratio r_i = g1_i / g0_i (Eq. (retention))
+ *                                  over the active coordinates
+ *   scale_mean                   : mean of scale_i (Eq. (scale_factor)); inactive
+ *                                  coordinates count with scale 1
+ *   disp_ratio                   : ||theta^{t,K} - theta^t|| / ||theta^{t,2} - theta^t||
+ *   inactive_frac                : 1 - |A_t| / n
+ * A coordinate whose ratio or scale is not a finite float32 is "irregular": it is
+ * counted in n_irregular and left out of the ratio, scale and displacement figures.
+ * With a caller-owned sum-of-squares buffer (gxpo_set_sumsq_buffer) gslow_norm and the
+ * cosine use whatever that buffer holds; everything else is this context's share. */
+typedef struct {
+    double g0_norm, g1_norm, gslow_norm, cos_g0_gslow, ratio_mean, ratio_std, scale_mean,
+           disp_ratio, inactive_frac;
+    long long n, n_active, n_irregular;
+} gxpo_diagnostics;
+
+/* Switch the diagnostics on or off; only legal between steps. */
+gxpo_status gxpo_enable_diagnostics(gxpo_ctx* ctx, int on);
+
+/* Diagnostics of the last completed active step.  Legal between steps, after an active
+ * step that ran with diagnostics on has gone through gxpo_gate_update.  Waits for
+ * `stream` (one small read-back).  Errors: STATE otherwise. */
+gxpo_status gxpo_get_diagnostics(gxpo_ctx* ctx, void* stream, gxpo_diagnostics* out);
+
 /* Host-side view of the gate, no device work. */
 gxpo_status gxpo_gate_peek(const gxpo_ctx* ctx, int* active, long long* s_star, long long* t);
 

@@ -54,6 +54,13 @@ class GateResult(ctypes.Structure):
                 ("mu", ctypes.c_double), ("sigma", ctypes.c_double)]
 
 
+class Diagnostics(ctypes.Structure):
+    _fields_ = [(k, ctypes.c_double) for k in
+                ("g0_norm", "g1_norm", "gslow_norm", "cos_g0_gslow", "ratio_mean", "ratio_std",
+                 "scale_mean", "disp_ratio", "inactive_frac")] + \
+               [(k, ctypes.c_longlong) for k in ("n", "n_active", "n_irregular")]
+
+
 _vp = ctypes.c_void_p
 _sigs = {
     "gxpo_default_cfg": (None, [ctypes.POINTER(Cfg), ctypes.POINTER(OptCfg)]),
@@ -68,6 +75,8 @@ _sigs = {
     "gxpo_slow_step": (ctypes.c_int, [_vp, _vp]),
     "gxpo_gate_update": (ctypes.c_int, [_vp, _vp, ctypes.POINTER(GateResult)]),
     "gxpo_set_sumsq_buffer": (ctypes.c_int, [_vp, _vp]),
+    "gxpo_enable_diagnostics": (ctypes.c_int, [_vp, ctypes.c_int]),
+    "gxpo_get_diagnostics": (ctypes.c_int, [_vp, _vp, ctypes.POINTER(Diagnostics)]),
     "gxpo_gate_peek": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_int),
                                       ctypes.POINTER(ctypes.c_longlong),
                                       ctypes.POINTER(ctypes.c_longlong)]),
@@ -210,6 +219,14 @@ class Context:
 
     def set_sumsq_buffer(self, dev_ptr: int):
         self._check(_lib.gxpo_set_sumsq_buffer(self._h, dev_ptr or None))
+
+    def enable_diagnostics(self, on: bool = True):
+        self._check(_lib.gxpo_enable_diagnostics(self._h, 1 if on else 0))
+
+    def get_diagnostics(self, stream=None) -> Diagnostics:
+        out = Diagnostics()
+        self._check(_lib.gxpo_get_diagnostics(self._h, _stream_ptr(stream), ctypes.byref(out)))
+        return out
 
     def gate_peek(self):
         a, s, t = ctypes.c_int(), ctypes.c_longlong(), ctypes.c_longlong()

@@ -63,6 +63,14 @@ struct gxpo_ctx {
     double* d_ring;
     GateResult* d_result;
     GateResult* h_result;              // pinned
+    // per-step diagnostics (off by default)
+    int diag_on;
+    int diag_ready;                    // 1 once an active step with diagnostics has completed
+    int gslow_aliased;                 // some tensor's g_slow shares g0's buffer: no <g0, g_slow>
+    double* d_diag;                    // kDiagN sums + <g0, g_slow>
+    double* d_diag_partials;           // kDiagN x kMaxGrid
+    DiagResult* d_diag_result;
+    DiagResult* h_diag_result;         // pinned
     // host mirror
     long long t, s_star, t_opt;
     long long launches;
@@ -181,8 +189,10 @@ StepParams make_step_params(gxpo_ctx* c, int which_grad, int in_sel, int out_sel
 
 typedef void (*StepFn)(const TensorDesc*, const ChunkRef*, long long, TensorDesc, StepParams, int,
                        double*, unsigned*, double*);
-typedef void (*ExtrapFn)(const TensorDesc*, const ChunkRef*, long long, TensorDesc, ExtrapParams, int);
-typedef void (*FusedFn)(const TensorDesc*, const ChunkRef*, long long, TensorDesc, FusedParams, int);
+typedef void (*ExtrapFn)(const TensorDesc*, const ChunkRef*, long long, TensorDesc, ExtrapParams, int,
+                         double*, unsigned*, double*);
+typedef void (*FusedFn)(const TensorDesc*, const ChunkRef*, long long, TensorDesc, FusedParams, int,
+                        double*, unsigned*, double*);
 
 StepFn pick_step(bool adamw, bool bf16, int variant) {
     if (variant == 1) {
@@ -192,21 +202,24 @@ StepFn pick_step(bool adamw, bool bf16, int variant) {
     if (adamw) return bf16 ? step_kernel<true, uint16_t, 8> : step_kernel<true, float, 8>;
     return bf16 ? step_kernel<false, uint16_t, 8> : step_kernel<false, float, 8>;
 }
-ExtrapFn pick_extrap(bool bf16, int variant) {
-    if (variant == 1) return bf16 ? extrap_kernel<uint16_t, 4> : extrap_kernel<float, 4>;
-    return bf16 ? extrap_kernel<uint16_t, 8> : extrap_kernel<float, 8>;
+// With diagnostics the sweeps use the 256-bit access variant only.
+ExtrapFn pick_extrap(bool bf16, int variant, bool diag) {
+    if (diag) return bf16 ? extrap_kernel<uint16_t, 8, true> : extrap_kernel<float, 8, true>;
+    if (variant == 1) return bf16 ? extrap_kernel<uint16_t, 4, false> : extrap_kernel<float, 4, false>;
+    return bf16 ? extrap_kernel<uint16_t, 8, false> : extrap_kernel<float, 8, false>;
 }
-template <bool DEFER>
+template <bool DEFER, bool DIAG>
 FusedFn pick_fused_t(bool adamw, bool bf16, int variant) {
-    if (variant == 1) {
-        if (adamw) return bf16 ? fused_kernel<true, uint16_t, 4, DEFER> : fused_kernel<true, float, 4, DEFER>;
-        return bf16 ? fused_kernel<false, uint16_t, 4, DEFER> : fused_kernel<false, float, 4, DEFER>;
+    if (variant == 1 && !DIAG) {
+        if (adamw) return bf16 ? fused_kernel<true, uint16_t, 4, DEFER, false> : fused_kernel<true, float, 4, DEFER, false>;
+        return bf16 ? fused_kernel<false, uint16_t, 4, DEFER, false> : fused_kernel<false, float, 4, DEFER, false>;
     }
-    if (adamw) return bf16 ? fused_kernel<true, uint16_t, 8, DEFER> : fused_kernel<true, float, 8, DEFER>;
-    return bf16 ? fused_kernel<false, uint16_t, 8, DEFER> : fused_kernel<false, float, 8, DEFER>;
+    if (adamw) return bf16 ? fused_kernel<true, uint16_t, 8, DEFER, DIAG> : fused_kernel<true, float, 8, DEFER, DIAG>;
+    return bf16 ? fused_kernel<false, uint16_t, 8, DEFER, DIAG> : fused_kernel<false, float, 8, DEFER, DIAG>;
 }
-FusedFn pick_fused(bool adamw, bool bf16, int variant, bool defer) {
-    return defer ? pick_fused_t<true>(adamw, bf16, variant) : pick_fused_t<false>(adamw, bf16, variant);
+FusedFn pick_fused(bool adamw, bool bf16, int variant, bool defer, bool diag) {
+    if (diag) return defer ? pick_fused_t<true, true>(adamw, bf16, variant) : pick_fused_t<false, true>(adamw, bf16, variant);
+    return defer ? pick_fused_t<true, false>(adamw, bf16, variant) : pick_fused_t<false, false>(adamw, bf16, variant);
 }
 
 // Launch one OptimStep sweep over either the bound list (chunks != null) or one
@@ -230,24 +243,31 @@ gxpo_status launch_step(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, co
 }
 
 gxpo_status launch_extrap(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
-                          long long num_chunks, const TensorDesc& flat, const ExtrapParams& p) {
-    if (num_chunks <= 0) return GXPO_OK;
-    ExtrapFn fn = pick_extrap(c->grad_dtype == GXPO_BF16, c->variant);
+                          long long num_chunks, const TensorDesc& flat, const ExtrapParams& p, bool diag) {
+    if (num_chunks <= 0) {
+        if (diag) CUDA_TRY(c, cudaMemsetAsync(c->d_diag, 0, (kDiagN + 1) * sizeof(double), s));
+        return GXPO_OK;
+    }
+    ExtrapFn fn = pick_extrap(c->grad_dtype == GXPO_BF16, c->variant, diag);
     const int ush = unit_shift_for(c, num_chunks);
     const int grid = grid_for(c, (const void*)fn, num_chunks << ush, kDefaultCtasExtrap);
-    fn<<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, ush);
+    fn<<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, ush, c->d_diag_partials, c->d_ticket, c->d_diag);
     c->launches += 1;
     CUDA_TRY(c, cudaGetLastError());
     return GXPO_OK;
 }
 
 gxpo_status launch_fused(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
-                         long long num_chunks, const TensorDesc& flat, const FusedParams& p, bool defer) {
-    if (num_chunks <= 0) return GXPO_OK;
-    FusedFn fn = pick_fused(c->opt.kind == GXPO_OPT_ADAMW, c->grad_dtype == GXPO_BF16, c->variant, defer);
+                         long long num_chunks, const TensorDesc& flat, const FusedParams& p, bool defer,
+                         bool diag) {
+    if (num_chunks <= 0) {
+        if (diag) CUDA_TRY(c, cudaMemsetAsync(c->d_diag, 0, (kDiagN + 1) * sizeof(double), s));
+        return GXPO_OK;
+    }
+    FusedFn fn = pick_fused(c->opt.kind == GXPO_OPT_ADAMW, c->grad_dtype == GXPO_BF16, c->variant, defer, diag);
     const int ush = unit_shift_for(c, num_chunks);
     const int grid = grid_for(c, (const void*)fn, num_chunks << ush, kDefaultCtasFused);
-    fn<<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, ush);
+    fn<<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, ush, c->d_diag_partials, c->d_ticket, c->d_diag);
     c->launches += 1;
     CUDA_TRY(c, cudaGetLastError());
     return GXPO_OK;
@@ -382,6 +402,11 @@ gxpo_status gxpo_create(const gxpo_cfg* cfg, const gxpo_opt_cfg* opt, int grad_d
     if (e == cudaSuccess) e = cudaMalloc(&c->d_ring, (size_t)cfg->window * sizeof(double));
     if (e == cudaSuccess) e = cudaMalloc(&c->d_result, sizeof(GateResult));
     if (e == cudaSuccess) e = cudaMallocHost(&c->h_result, sizeof(GateResult));
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_diag, (kDiagN + 1) * sizeof(double));
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_diag_partials, (size_t)kDiagN * kMaxGrid * sizeof(double));
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_diag_result, sizeof(DiagResult));
+    if (e == cudaSuccess) e = cudaMallocHost(&c->h_diag_result, sizeof(DiagResult));
+    if (e == cudaSuccess) e = cudaMemset(c->d_diag, 0, (kDiagN + 1) * sizeof(double));
     if (e == cudaSuccess) e = cudaMemset(c->d_ticket, 0, sizeof(unsigned));
     if (e == cudaSuccess) e = cudaMemset(c->d_sumsq, 0, sizeof(double));
     if (e == cudaSuccess) e = cudaMemset(c->d_ring, 0, (size_t)cfg->window * sizeof(double));
@@ -410,6 +435,10 @@ void gxpo_destroy(gxpo_ctx* c) {
     cudaFree(c->d_ring);
     cudaFree(c->d_result);
     if (c->h_result) cudaFreeHost(c->h_result);
+    cudaFree(c->d_diag);
+    cudaFree(c->d_diag_partials);
+    cudaFree(c->d_diag_result);
+    if (c->h_diag_result) cudaFreeHost(c->h_diag_result);
     delete c;
 }
 
@@ -436,6 +465,7 @@ gxpo_status gxpo_bind(gxpo_ctx* c, const gxpo_tensor* list, int count) {
     std::vector<TensorDesc> descs((size_t)count);
     std::vector<ChunkRef> chunks;
     long long total = 0;
+    int aliased = 0;
     for (int i = 0; i < count; ++i) {
         gxpo_status s = check_tensor(c, list[i], i, true);
         if (s != GXPO_OK) return s;
@@ -444,6 +474,7 @@ gxpo_status gxpo_bind(gxpo_ctx* c, const gxpo_tensor* list, int count) {
         d.g[0] = list[i].g0; d.g[1] = list[i].g1; d.g[2] = list[i].g_slow;
         d.n = list[i].n;
         total += d.n;
+        if (d.n > 0 && d.g[2] == d.g[0]) aliased = 1;
     }
     chunks.reserve((size_t)(total / kChunk + count));
     for (int i = 0; i < count; ++i) {
@@ -465,6 +496,8 @@ gxpo_status gxpo_bind(gxpo_ctx* c, const gxpo_tensor* list, int count) {
     c->num_chunks = (long long)chunks.size();
     c->num_tensors = count;
     c->total_params = total;
+    c->gslow_aliased = aliased;
+    c->diag_ready = 0;
     c->bound = 1;
     return GXPO_OK;
 }
@@ -529,7 +562,7 @@ gxpo_status gxpo_extrapolate(gxpo_ctx* c, void* stream) {
     if (c->phase != PROBED1) return fail(c, GXPO_ERR_STATE, "extrapolate must follow probe step 1");
     const TensorDesc none = {};
     gxpo_status st = launch_extrap(c, (cudaStream_t)stream, c->d_descs, c->d_chunks, c->num_chunks, none,
-                                   make_extrap_params(c, c->cfg.placement));
+                                   make_extrap_params(c, c->cfg.placement), c->diag_on != 0);
     if (st != GXPO_OK) return st;
     c->phase = EXTRAPOLATED;
     return GXPO_OK;
@@ -547,7 +580,8 @@ gxpo_status gxpo_probe_extrapolate(gxpo_ctx* c, void* stream) {
     c->t_opt += 1;
     p.step = (place == GXPO_PLACE_PINGPONG) ? make_step_params(c, 1, 1, 1, 0, 0) : make_step_params(c, 1, 0, 0, 0, 0);
     p.ex = make_extrap_params(c, place);
-    gxpo_status st = launch_fused(c, (cudaStream_t)stream, c->d_descs, c->d_chunks, c->num_chunks, none, p, defer);
+    gxpo_status st = launch_fused(c, (cudaStream_t)stream, c->d_descs, c->d_chunks, c->num_chunks, none, p, defer,
+                                  c->diag_on != 0);
     if (st != GXPO_OK) { c->t_opt -= 1; return st; }
     c->phase = EXTRAPOLATED;
     return GXPO_OK;
@@ -562,6 +596,15 @@ gxpo_status gxpo_slow_step(gxpo_ctx* c, void* stream) {
     gxpo_status st = launch_step(c, (cudaStream_t)stream, c->d_descs, c->d_chunks, c->num_chunks, none, p,
                                  c->user_sumsq ? c->user_sumsq : c->d_sumsq);
     if (st != GXPO_OK) { c->t_opt -= 1; return st; }
+    if (c->diag_on && !c->gslow_aliased && c->num_chunks > 0) {
+        const bool bf16 = c->grad_dtype == GXPO_BF16;
+        long long g = (long long)c->sm_count * 4;
+        if (g > c->num_chunks) g = c->num_chunks;
+        if (bf16) dot_kernel<uint16_t><<<(int)g, kThreads, 0, (cudaStream_t)stream>>>(c->d_descs, c->d_chunks, c->num_chunks, c->d_partials, c->d_ticket, c->d_diag + kDiagN);
+        else      dot_kernel<float><<<(int)g, kThreads, 0, (cudaStream_t)stream>>>(c->d_descs, c->d_chunks, c->num_chunks, c->d_partials, c->d_ticket, c->d_diag + kDiagN);
+        c->launches += 1;
+        CUDA_TRY(c, cudaGetLastError());
+    }
     c->phase = SLOW_DONE;
     return GXPO_OK;
 }
@@ -570,6 +613,7 @@ gxpo_status gxpo_gate_update(gxpo_ctx* c, void* stream, gxpo_gate_result* out) {
     if (!c) return GXPO_ERR_INVALID_ARG;
     if (c->phase != SLOW_DONE) return fail(c, GXPO_ERR_STATE, "gate update must follow the slow step");
     c->phase = IDLE;
+    c->diag_ready = c->diag_on;
     return run_gate(c, (cudaStream_t)stream, c->user_sumsq ? c->user_sumsq : c->d_sumsq, out);
 }
 
@@ -578,6 +622,33 @@ gxpo_status gxpo_set_sumsq_buffer(gxpo_ctx* c, double* sumsq_dev) {
     if (c->phase == SLOW_DONE) return fail(c, GXPO_ERR_STATE, "a norm is pending: call gxpo_gate_update first");
     if (((uintptr_t)sumsq_dev) & 7u) return fail(c, GXPO_ERR_ALIGNMENT, "sumsq buffer must be 8-byte aligned");
     c->user_sumsq = sumsq_dev;
+    return GXPO_OK;
+}
+
+gxpo_status gxpo_enable_diagnostics(gxpo_ctx* c, int on) {
+    if (!c) return GXPO_ERR_INVALID_ARG;
+    if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "diagnostics can only be switched between steps");
+    c->diag_on = on ? 1 : 0;
+    c->diag_ready = 0;
+    return GXPO_OK;
+}
+
+gxpo_status gxpo_get_diagnostics(gxpo_ctx* c, void* stream, gxpo_diagnostics* out) {
+    if (!c || !out) return GXPO_ERR_INVALID_ARG;
+    if (c->phase != IDLE || !c->diag_ready)
+        return fail(c, GXPO_ERR_STATE, "no diagnostics: enable them, then complete an active step through gxpo_gate_update");
+    cudaStream_t s = (cudaStream_t)stream;
+    diag_finalize_kernel<<<1, 32, 0, s>>>(c->d_diag, c->user_sumsq ? c->user_sumsq : c->d_sumsq, c->total_params,
+                                          c->gslow_aliased ? 0 : 1, c->d_diag_result);
+    c->launches += 1;
+    CUDA_TRY(c, cudaGetLastError());
+    CUDA_TRY(c, cudaMemcpyAsync(c->h_diag_result, c->d_diag_result, sizeof(DiagResult), cudaMemcpyDeviceToHost, s));
+    CUDA_TRY(c, cudaStreamSynchronize(s));
+    const DiagResult r = *c->h_diag_result;
+    out->g0_norm = r.g0_norm; out->g1_norm = r.g1_norm; out->gslow_norm = r.gslow_norm;
+    out->cos_g0_gslow = r.cos_g0_gslow; out->ratio_mean = r.ratio_mean; out->ratio_std = r.ratio_std;
+    out->scale_mean = r.scale_mean; out->disp_ratio = r.disp_ratio; out->inactive_frac = r.inactive_frac;
+    out->n = r.n; out->n_active = r.n_active; out->n_irregular = r.n_irregular;
     return GXPO_OK;
 }
 
@@ -739,7 +810,7 @@ gxpo_status gxpo_step_host(gxpo_ctx* c, const gxpo_tensor* list, int count, long
                 fp.step0 = make_step_params(c, 0, 0, 0, 0, 0);
                 fp.step = make_step_params(c, 1, 1, 1, 0, 0);
                 fp.ex = make_extrap_params(c, GXPO_PLACE_PINGPONG);
-                rs = launch_fused(c, s, nullptr, nullptr, nch, d, fp, false);
+                rs = launch_fused(c, s, nullptr, nullptr, nch, d, fp, false, false);
                 if (rs != GXPO_OK) return rs;
                 c->t_opt = t_opt0 + 3;
                 rs = launch_step(c, s, nullptr, nullptr, nch, d, make_step_params(c, 2, 0, 0, 0, 1), st.piece_sumsq + 1);
