@@ -197,6 +197,25 @@ gxpo_status gxpo_gate_update(gxpo_ctx* ctx, void* stream, gxpo_gate_result* out)
  * same reduced value on every rank the gates flip together. */
 gxpo_status gxpo_set_sumsq_buffer(gxpo_ctx* ctx, double* sumsq_dev);
 
+/* Gradient scaling and global-norm clipping (the paper's training recipe clips at 1.0;
+ * it is the trainer's step, not part of Algorithm 1).  A scale is a DEVICE float that
+ * every sweep multiplies into gradient `which` (0 = g0, 1 = g1, 2 = g_slow) as it loads
+ * it: the optimizer steps and the retention ratio see the scaled gradient, while
+ * ||g_slow|| for the gate is taken of the gradient as given.  NULL = no scaling.
+ * Only legal between steps. */
+gxpo_status gxpo_set_grad_scale(gxpo_ctx* ctx, int which, const float* scale_dev);
+
+/* Clip gradient `which` by its global norm over the bound list: one pass over that
+ * gradient computes ||g||, a device-side step turns it into min(1, max_norm / (||g|| + 1e-6))
+ * (the usual trainers' convention), and the sweeps of THIS training step scale the
+ * gradient by it as they load it -- the gradient buffer itself is not rewritten, so
+ * clipping costs one read of g instead of a read plus a read-modify-write.  Call it
+ * right before the sweep that consumes the gradient (which = 0 before the first probe
+ * or fallback step, 1 before the second probe, 2 before the slow step); the coefficient
+ * expires at the end of the step.  Asynchronous on `stream`.
+ * Errors: STATE at any other point of the call order, INVALID_ARG for max_norm <= 0. */
+gxpo_status gxpo_clip_grad_norm(gxpo_ctx* ctx, int which, double max_norm, void* stream);
+
 /* Per-step diagnostics of the active phase: the quantities the paper's appendix
  * tabulates ("Active-phase GXPO diagnostics").  Off by default.  When on, the sums are
  * gathered inside the extrapolation sweep (gxpo_extrapolate or gxpo_probe_extrapolate) at

@@ -133,6 +133,15 @@ double gxo_sum_squares(const double* g, int64_t n) {
 
 double gxo_l2norm(const double* g, int64_t n) { return std::sqrt(gxo_sum_squares(g, n)); }
 
+/* ---- Global-norm gradient clipping (the paper's recipe: "gradient clipping at 1.0";
+ *      a trainer step, not part of Algorithm 1).  The paper gives no formula; this is
+ *      the trainers' usual one: every gradient is multiplied by
+ *      min(1, max_norm / (||g||_2 + 1e-6)). */
+double gxo_clip_coef(double norm, double max_norm) {
+    const double c = max_norm / (norm + 1e-6);
+    return c < 1.0 ? c : 1.0;
+}
+
 /* ---- Per-step diagnostics of the active phase, the quantities the paper's appendix
  *      tabulates ("Active-phase GXPO diagnostics": gradient norms, cos(g0, g_slow),
  *      retention ratio mean +- std, ||Delta_K|| / ||Delta_2||, scale mean, inactive

@@ -54,6 +54,8 @@ def lib():
         L.gxo_sum_squares.restype = ctypes.c_double
         L.gxo_l2norm.argtypes = [_f64p, _i64]
         L.gxo_l2norm.restype = ctypes.c_double
+        L.gxo_clip_coef.argtypes = [ctypes.c_double, ctypes.c_double]
+        L.gxo_clip_coef.restype = ctypes.c_double
         L.gxo_active_diagnostics.argtypes = [_f64p] * 5 + [_i64, ctypes.c_int, ctypes.c_double,
                                              ctypes.c_double, _f64p]
         L.gxo_active_diagnostics.restype = None
@@ -145,6 +147,11 @@ def sum_squares(g) -> float:
 
 def l2norm(g) -> float:
     return float(lib().gxo_l2norm(_p(g), g.size))
+
+
+def clip_coef(norm: float, max_norm: float) -> float:
+    """min(1, max_norm / (norm + 1e-6)): the global-norm clipping coefficient."""
+    return float(lib().gxo_clip_coef(float(norm), float(max_norm)))
 
 
 DIAG_FIELDS = ("g0_norm", "g1_norm", "gslow_norm", "cos_g0_gslow", "ratio_mean", "ratio_std",

@@ -75,6 +75,8 @@ _sigs = {
     "gxpo_slow_step": (ctypes.c_int, [_vp, _vp]),
     "gxpo_gate_update": (ctypes.c_int, [_vp, _vp, ctypes.POINTER(GateResult)]),
     "gxpo_set_sumsq_buffer": (ctypes.c_int, [_vp, _vp]),
+    "gxpo_set_grad_scale": (ctypes.c_int, [_vp, ctypes.c_int, _vp]),
+    "gxpo_clip_grad_norm": (ctypes.c_int, [_vp, ctypes.c_int, ctypes.c_double, _vp]),
     "gxpo_enable_diagnostics": (ctypes.c_int, [_vp, ctypes.c_int]),
     "gxpo_get_diagnostics": (ctypes.c_int, [_vp, _vp, ctypes.POINTER(Diagnostics)]),
     "gxpo_gate_peek": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_int),
@@ -219,6 +221,12 @@ class Context:
 
     def set_sumsq_buffer(self, dev_ptr: int):
         self._check(_lib.gxpo_set_sumsq_buffer(self._h, dev_ptr or None))
+
+    def set_grad_scale(self, which: int, scale_ptr: int):
+        self._check(_lib.gxpo_set_grad_scale(self._h, which, scale_ptr or None))
+
+    def clip_grad_norm(self, which: int, max_norm: float, stream=None):
+        self._check(_lib.gxpo_clip_grad_norm(self._h, which, max_norm, _stream_ptr(stream)))
 
     def enable_diagnostics(self, on: bool = True):
         self._check(_lib.gxpo_enable_diagnostics(self._h, 1 if on else 0))

@@ -64,6 +64,11 @@ struct gxpo_ctx {
     GateResult* d_result;
     GateResult* h_result;              // pinned
     // per-step diagnostics (off by default)
+    // gradient scaling: per gradient a device scalar (caller's, or clip[] below), or null
+    const float* gscale[3];            // what the sweeps use
+    const float* user_gscale[3];       // what gxpo_set_grad_scale gave (restored when a clip expires)
+    float* d_clip;                     // [3] clipping coefficients written by gxpo_clip_grad_norm
+    double* d_gnorm;                   // [3] sum of squares, then [3] norms, of the clipped gradients
     int diag_on;
     int diag_ready;                    // 1 once an active step with diagnostics has completed
     int gslow_aliased;                 // some tensor's g_slow shares g0's buffer: no <g0, g_slow>
@@ -169,6 +174,7 @@ StepParams make_step_params(gxpo_ctx* c, int which_grad, int in_sel, int out_sel
     p.snapshot = snapshot;
     p.want_norm = want_norm;
     p.write_state = 1;
+    p.gscale = c->gscale[which_grad];
     const gxpo_opt_cfg& o = c->opt;
     p.lr = (float)o.lr;
     if (o.kind == GXPO_OPT_ADAMW) {
@@ -279,12 +285,19 @@ ExtrapParams make_extrap_params(const gxpo_ctx* c, int placement) {
     p.alpha = c->cfg.alpha;
     p.delta = c->cfg.delta;
     p.den_eps = c->cfg.den_eps;
+    p.gscale0 = c->gscale[0];
+    p.gscale1 = c->gscale[1];
     if (placement == GXPO_PLACE_PINGPONG) { p.theta2_sel = 1; p.theta0_sel = 0; }
     else { p.theta2_sel = 0; p.theta0_sel = 1; }
     return p;
 }
 
 bool gate_active(const gxpo_ctx* c) { return c->s_star < 0 || c->t < c->s_star; }
+
+// A clipping coefficient belongs to the step it was computed in.
+void expire_clips(gxpo_ctx* c) {
+    for (int k = 0; k < 3; ++k) c->gscale[k] = c->user_gscale[k];
+}
 
 gxpo_status run_gate(gxpo_ctx* c, cudaStream_t s, const double* sumsq, gxpo_gate_result* out) {
     gate_kernel<<<1, 32, 0, s>>>(c->d_gate, c->d_ring, sumsq, c->t, c->cfg.tau, c->cfg.gate_eps,
@@ -402,6 +415,8 @@ gxpo_status gxpo_create(const gxpo_cfg* cfg, const gxpo_opt_cfg* opt, int grad_d
     if (e == cudaSuccess) e = cudaMalloc(&c->d_ring, (size_t)cfg->window * sizeof(double));
     if (e == cudaSuccess) e = cudaMalloc(&c->d_result, sizeof(GateResult));
     if (e == cudaSuccess) e = cudaMallocHost(&c->h_result, sizeof(GateResult));
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_clip, 3 * sizeof(float));
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_gnorm, 6 * sizeof(double));
     if (e == cudaSuccess) e = cudaMalloc(&c->d_diag, (kDiagN + 1) * sizeof(double));
     if (e == cudaSuccess) e = cudaMalloc(&c->d_diag_partials, (size_t)kDiagN * kMaxGrid * sizeof(double));
     if (e == cudaSuccess) e = cudaMalloc(&c->d_diag_result, sizeof(DiagResult));
@@ -435,6 +450,8 @@ void gxpo_destroy(gxpo_ctx* c) {
     cudaFree(c->d_ring);
     cudaFree(c->d_result);
     if (c->h_result) cudaFreeHost(c->h_result);
+    cudaFree(c->d_clip);
+    cudaFree(c->d_gnorm);
     cudaFree(c->d_diag);
     cudaFree(c->d_diag_partials);
     cudaFree(c->d_diag_result);
@@ -516,6 +533,7 @@ gxpo_status gxpo_probe_step(gxpo_ctx* c, int which, void* stream) {
         gxpo_status st = launch_step(c, s, c->d_descs, c->d_chunks, c->num_chunks, none, p, c->d_sumsq);
         if (st != GXPO_OK) { c->t_opt -= 1; return st; }
         c->t += 1;
+        expire_clips(c);
         return GXPO_OK;
     }
     if (which == 0) {
@@ -600,8 +618,8 @@ gxpo_status gxpo_slow_step(gxpo_ctx* c, void* stream) {
         const bool bf16 = c->grad_dtype == GXPO_BF16;
         long long g = (long long)c->sm_count * 4;
         if (g > c->num_chunks) g = c->num_chunks;
-        if (bf16) dot_kernel<uint16_t><<<(int)g, kThreads, 0, (cudaStream_t)stream>>>(c->d_descs, c->d_chunks, c->num_chunks, c->d_partials, c->d_ticket, c->d_diag + kDiagN);
-        else      dot_kernel<float><<<(int)g, kThreads, 0, (cudaStream_t)stream>>>(c->d_descs, c->d_chunks, c->num_chunks, c->d_partials, c->d_ticket, c->d_diag + kDiagN);
+        if (bf16) dot_kernel<uint16_t><<<(int)g, kThreads, 0, (cudaStream_t)stream>>>(c->d_descs, c->d_chunks, c->num_chunks, 0, 2, c->d_partials, c->d_ticket, c->d_diag + kDiagN);
+        else      dot_kernel<float><<<(int)g, kThreads, 0, (cudaStream_t)stream>>>(c->d_descs, c->d_chunks, c->num_chunks, 0, 2, c->d_partials, c->d_ticket, c->d_diag + kDiagN);
         c->launches += 1;
         CUDA_TRY(c, cudaGetLastError());
     }
@@ -614,6 +632,7 @@ gxpo_status gxpo_gate_update(gxpo_ctx* c, void* stream, gxpo_gate_result* out) {
     if (c->phase != SLOW_DONE) return fail(c, GXPO_ERR_STATE, "gate update must follow the slow step");
     c->phase = IDLE;
     c->diag_ready = c->diag_on;
+    expire_clips(c);
     return run_gate(c, (cudaStream_t)stream, c->user_sumsq ? c->user_sumsq : c->d_sumsq, out);
 }
 
@@ -622,6 +641,46 @@ gxpo_status gxpo_set_sumsq_buffer(gxpo_ctx* c, double* sumsq_dev) {
     if (c->phase == SLOW_DONE) return fail(c, GXPO_ERR_STATE, "a norm is pending: call gxpo_gate_update first");
     if (((uintptr_t)sumsq_dev) & 7u) return fail(c, GXPO_ERR_ALIGNMENT, "sumsq buffer must be 8-byte aligned");
     c->user_sumsq = sumsq_dev;
+    return GXPO_OK;
+}
+
+gxpo_status gxpo_set_grad_scale(gxpo_ctx* c, int which, const float* scale_dev) {
+    if (!c) return GXPO_ERR_INVALID_ARG;
+    if (which < 0 || which > 2) return fail(c, GXPO_ERR_INVALID_ARG, "which must be 0 (g0), 1 (g1) or 2 (g_slow)");
+    if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "gradient scales can only be changed between steps");
+    if (((uintptr_t)scale_dev) & 3u) return fail(c, GXPO_ERR_ALIGNMENT, "scale pointer must be 4-byte aligned");
+    c->gscale[which] = scale_dev;
+    c->user_gscale[which] = scale_dev;
+    return GXPO_OK;
+}
+
+gxpo_status gxpo_clip_grad_norm(gxpo_ctx* c, int which, double max_norm, void* stream) {
+    if (!c) return GXPO_ERR_INVALID_ARG;
+    if (which < 0 || which > 2) return fail(c, GXPO_ERR_INVALID_ARG, "which must be 0 (g0), 1 (g1) or 2 (g_slow)");
+    if (!(max_norm > 0.0) || !std::isfinite(max_norm)) return fail(c, GXPO_ERR_INVALID_ARG, "max_norm must be finite and > 0");
+    if (!c->bound) return fail(c, GXPO_ERR_STATE, "nothing bound: call gxpo_bind first");
+    // legal exactly where the sweep that consumes this gradient is the next one to run
+    const bool ok = (which == 0 && c->phase == IDLE) ||
+                    (which == 1 && (c->phase == PROBED0 || c->phase == PROBED0_DEFERRED)) ||
+                    (which == 2 && c->phase == EXTRAPOLATED);
+    if (!ok) return fail(c, GXPO_ERR_STATE, "clip the gradient right before the sweep that consumes it");
+    cudaStream_t s = (cudaStream_t)stream;
+    if (c->num_chunks > 0) {
+        long long g = (long long)c->sm_count * 4;
+        if (g > c->num_chunks) g = c->num_chunks;
+        if (c->grad_dtype == GXPO_BF16)
+            dot_kernel<uint16_t><<<(int)g, kThreads, 0, s>>>(c->d_descs, c->d_chunks, c->num_chunks, which, which, c->d_partials, c->d_ticket, c->d_gnorm + which);
+        else
+            dot_kernel<float><<<(int)g, kThreads, 0, s>>>(c->d_descs, c->d_chunks, c->num_chunks, which, which, c->d_partials, c->d_ticket, c->d_gnorm + which);
+        c->launches += 1;
+        CUDA_TRY(c, cudaGetLastError());
+    } else {
+        CUDA_TRY(c, cudaMemsetAsync(c->d_gnorm + which, 0, sizeof(double), s));
+    }
+    clip_coef_kernel<<<1, 32, 0, s>>>(c->d_gnorm + which, max_norm, c->d_clip + which, c->d_gnorm + 3 + which);
+    c->launches += 1;
+    CUDA_TRY(c, cudaGetLastError());
+    c->gscale[which] = c->d_clip + which;
     return GXPO_OK;
 }
 
@@ -914,8 +973,8 @@ step_flat_perchunk_kernel(TensorDesc d, long long num_chunks, StepParams p, doub
         const G* g = reinterpret_cast<const G*>(d.g[2]) + off;
         const bool vec = aligned32(th) && aligned32(g) && (!ADAMW || (aligned32(m) && aligned32(v)));
         double acc = 0.0;
-        if (vec) step_chunk_vec<ADAMW, G, 8>(th, th, nullptr, m, v, g, len, p, acc);
-        else     step_chunk_scalar<ADAMW, G>(th, th, nullptr, m, v, g, len, p, acc);
+        if (vec) step_chunk_vec<ADAMW, G, 8>(th, th, nullptr, m, v, g, len, p, 1.0f, acc);
+        else     step_chunk_scalar<ADAMW, G>(th, th, nullptr, m, v, g, len, p, 1.0f, acc);
         const double tot = block_sum(acc, red);
         if (threadIdx.x == 0) partials[c] = tot;
     }

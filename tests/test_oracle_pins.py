@@ -250,3 +250,22 @@ def test_bf16_conversion_helpers_are_exact():
     tie = np.array([1.0 + 2.0**-8, 1.0 + 3 * 2.0**-8], dtype=np.float32)
     np.testing.assert_array_equal(workloads.bf16_bits_to_f32(workloads.f32_to_bf16_bits(tie)),
                                   np.array([1.0, 1.0 + 2.0**-6], dtype=np.float32))
+
+
+def test_clip_coefficient_matches_the_library_routine():
+    """Global-norm clipping against torch.nn.utils.clip_grad_norm_ (float64, CPU)."""
+    import torch
+    rng = np.random.default_rng(11)
+    for scale, max_norm in [(1.0, 1.0), (1e-3, 1.0), (5.0, 0.3), (1.0, 100.0)]:
+        gs = [scale * rng.standard_normal(n) for n in (7, 100, 1)]
+        ps = [torch.nn.Parameter(torch.zeros(g.size, dtype=torch.float64)) for g in gs]
+        for p, g in zip(ps, gs):
+            p.grad = torch.from_numpy(g.copy())
+        total = float(torch.nn.utils.clip_grad_norm_(ps, max_norm))
+        norm = math.sqrt(sum(ora.sum_squares(np.ascontiguousarray(g)) for g in gs))
+        assert norm == pytest.approx(total, rel=1e-14)
+        c = ora.clip_coef(norm, max_norm)
+        for p, g in zip(ps, gs):
+            np.testing.assert_allclose(p.grad.numpy(), g * c, rtol=1e-14, atol=0)
+        assert (c == 1.0) == (max_norm / (norm + 1e-6) >= 1.0)
+    assert ora.clip_coef(0.0, 1.0) == 1.0 and ora.clip_coef(2.0, 1.0) == pytest.approx(1 / (2 + 1e-6), rel=1e-15)
