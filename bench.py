@@ -63,6 +63,9 @@ def parse_args():
     ap.add_argument("--flow", default="deferred", choices=["deferred", "fused", "unfused"],
                     help="deferred: probe_step_deferred + probe_extrapolate (72 B/param, default); "
                          "fused: probe_step(0) + probe_extrapolate (84); unfused: the four separate sweeps (94)")
+    ap.add_argument("--emit-bf16", action="store_true",
+                    help="also keep bfloat16 model-weight copies (gxpo_bind_model_weights, bf16-only theta1): "
+                         "16 + 30 + 28 = 74 B/param, and the caller needs no cast sweeps")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-params", type=int, default=1 << 26)
@@ -250,15 +253,15 @@ def build_device_workload(torch, b, shapes, seed, alias_gslow):
     return d, ptrs, (theta, work, m, v, g0, g1, gs)
 
 
-def plan_workload(args, free_bytes, margin=6 << 30):
+def plan_workload(args, free_bytes, margin=6 << 30, extra_bytes=0):
     """Shapes of the workload and whether g_slow has to share g0's buffer (legal: g0 is
     dead once the extrapolation has run) so that 22 -> 20 bytes per parameter fit into
     the free device memory; as a last resort the decoder depth is reduced, and the
     description says so."""
     shapes, desc = workload_shapes(args)
     d = sum(k for _, k in shapes)
-    alias = 22 * d + margin > free_bytes
-    while (20 if alias else 22) * d + margin > free_bytes and args.workload in ("qwen25_7b", "llama31_8b"):
+    alias = (22 + extra_bytes) * d + margin > free_bytes
+    while ((20 if alias else 22) + extra_bytes) * d + margin > free_bytes and args.workload in ("qwen25_7b", "llama31_8b"):
         args.layers = (args.layers or (28 if args.workload == "qwen25_7b" else 32)) - 1
         if args.layers < 1:
             raise SystemExit("not enough free device memory for even one decoder layer")
@@ -288,7 +291,8 @@ def run_ours(args):
     stream = torch.cuda.current_stream()
 
     free, total = torch.cuda.mem_get_info()
-    shapes, desc, alias = plan_workload(args, free)
+    emit = bool(getattr(args, "emit_bf16", False)) and args.flow == "deferred" and not args.fallback
+    shapes, desc, alias = plan_workload(args, free, extra_bytes=2 if emit else 0)
     d, ptrs, keep = build_device_workload(torch, b, shapes, 1000 + rank, alias)
     sumsq = torch.zeros(1, dtype=torch.float64, device="cuda")
 
@@ -296,6 +300,13 @@ def run_ours(args):
     ctx = b.Context(cfg, opt, b.BF16)
     ctx.tune(args.ctas, args.variant, args.unit_tiles)
     ctx.bind(ptrs)
+    if emit:
+        weights = torch.empty(d, dtype=torch.bfloat16, device="cuda")
+        offs, acc = [], 0
+        for _, k in shapes:
+            offs.append(acc)
+            acc += k
+        ctx.bind_model_weights([weights.data_ptr() + 2 * o for o in offs], only_bf16_theta1=True)
     if world > 1:
         ctx.set_sumsq_buffer(sumsq.data_ptr())
 
@@ -376,6 +387,10 @@ def run_ours(args):
                  "probe_step1": BYTES_STEP_ADAMW, "extrapolate": BYTES_EXTRAP,
                  "probe_extrapolate": BYTES_FUSED, "probe_extrapolate_deferred": BYTES_FUSED_DEFERRED,
                  "slow_step": BYTES_STEP_ADAMW, "fallback_step": BYTES_STEP_ADAMW}
+    if emit:      # bf16 copies: theta1 as bf16 only (-4 + 2), theta-tilde and theta_new also as bf16 (+2 each)
+        alg_bytes["probe_step0_deferred"] -= 2
+        alg_bytes["probe_extrapolate_deferred"] += 2
+        alg_bytes["slow_step"] += 2
     kernels = {nm: {"kernel": KERNEL_OF[nm], "ms": ms, "bytes_per_param": alg_bytes[nm],
                     "gbs": alg_bytes[nm] * d / (ms * 1e-3) / 1e9} for nm, ms in per.items()}
     # dominant kernel = the kernel function with the largest share of the step; its figures
@@ -409,7 +424,7 @@ def run_ours(args):
                    {"deferred": "active (probe with deferred state, probe+extrapolate in one sweep, slow step, gate)",
                     "fused": "active (probe, probe+extrapolate in one sweep, slow step, gate)",
                     "unfused": "active (probe, probe, extrapolate, slow step, gate)"}[flow],
-                   "g_slow_aliases_g0": alias, "l2": "inputs larger than L2 (no flush needed)",
+                   "bf16_model_weight_copies": emit, "g_slow_aliases_g0": alias, "l2": "inputs larger than L2 (no flush needed)",
                    "parallelism": f"dp{world} (independent shards, one 8-byte all-reduce per step)" if world > 1 else "1 GPU"},
         "hbm_gbs_whole_step": whole_gbs, "hbm_frac_whole_step": whole_gbs / peak,
         "hbm_frac_of_8tbs_nominal": whole_gbs / 8000.0,

@@ -138,6 +138,23 @@ void gxpo_destroy(gxpo_ctx* ctx);
  * AdamW), ALIGNMENT (pointer not aligned to its element size), STATE (mid-step). */
 gxpo_status gxpo_bind(gxpo_ctx* ctx, const gxpo_tensor* list, int count);
 
+/* Optional bfloat16 copies of the live parameters, for trainers whose model runs its
+ * forward and backward passes on bfloat16 weights while this library keeps the float32
+ * masters (the paper trains in bf16).  weights_bf16[i] is a DEVICE buffer of the i-th
+ * bound tensor's length (or NULL for none); count must equal the bound count.  Every
+ * sweep that produces a point a backward pass is taken at -- the first probe step
+ * (theta^{t,1}), the extrapolation (theta-tilde), the slow step and the fallback step
+ * (theta^{t+1}) -- then also stores that point rounded to nearest-even bfloat16, which
+ * saves the caller a separate cast sweep (read 4 + write 2 bytes per parameter) before
+ * each backward pass.  The second probe step's point is never needed and not stored.
+ * only_bf16_theta1 != 0: gxpo_probe_step_deferred writes ONLY the bfloat16 copy of
+ * theta^{t,1} (gxpo_probe_extrapolate recomputes the float32 value anyway), so `work` is
+ * left untouched; needs PINGPONG placement and a buffer for every non-empty tensor.
+ * Pass weights_bf16 = NULL to unbind.  gxpo_bind drops the binding.  Only legal between
+ * steps; waits for the device. */
+gxpo_status gxpo_bind_model_weights(gxpo_ctx* ctx, void* const* weights_bf16, int count,
+                                    int only_bf16_theta1);
+
 /* Algorithm 1, "first/second fast optimizer step" (which = 0, 1) and the fallback
  * phase's single step (which = -1).
  *   which =  0: theta^{t,1} <- OptimStep(theta^t, g0)      state: IDLE   -> PROBED0

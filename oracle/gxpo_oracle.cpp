@@ -32,6 +32,7 @@
 #include <cmath>
 #include <cstdint>
 #include <cstdlib>
+#include <cstring>
 #include <limits>
 
 namespace {
@@ -132,6 +133,25 @@ double gxo_sum_squares(const double* g, int64_t n) {
 }
 
 double gxo_l2norm(const double* g, int64_t n) { return std::sqrt(gxo_sum_squares(g, n)); }
+
+/* ---- float32 -> bfloat16, round to nearest even: the model-weight copy a bf16 trainer
+ *      runs its forward and backward passes on (the paper trains in bf16; the master
+ *      parameters here are fp32).  bfloat16 is the upper 16 bits of the float32 pattern;
+ *      rounding adds half of the dropped field, ties to the even 16-bit pattern; a NaN
+ *      stays a (quiet) NaN.  Returns the 16-bit pattern. */
+uint16_t gxo_f32_to_bf16(float x) {
+    uint32_t u;
+    std::memcpy(&u, &x, sizeof(u));
+    if ((u & 0x7fffffffu) > 0x7f800000u) return static_cast<uint16_t>((u >> 16) | 0x0040u);
+    const uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7fffu + lsb;
+    return static_cast<uint16_t>(u >> 16);
+}
+
+/* theta (double holding float32 values) -> bfloat16 patterns, element by element */
+void gxo_round_to_bf16(const double* theta, uint16_t* out, int64_t n) {
+    for (int64_t i = 0; i < n; ++i) out[i] = gxo_f32_to_bf16(static_cast<float>(theta[i]));
+}
 
 /* ---- Global-norm gradient clipping (the paper's recipe: "gradient clipping at 1.0";
  *      a trainer step, not part of Algorithm 1).  The paper gives no formula; this is

@@ -54,6 +54,8 @@ def lib():
         L.gxo_sum_squares.restype = ctypes.c_double
         L.gxo_l2norm.argtypes = [_f64p, _i64]
         L.gxo_l2norm.restype = ctypes.c_double
+        L.gxo_round_to_bf16.argtypes = [_f64p, ctypes.POINTER(ctypes.c_uint16), _i64]
+        L.gxo_round_to_bf16.restype = None
         L.gxo_clip_coef.argtypes = [ctypes.c_double, ctypes.c_double]
         L.gxo_clip_coef.restype = ctypes.c_double
         L.gxo_active_diagnostics.argtypes = [_f64p] * 5 + [_i64, ctypes.c_int, ctypes.c_double,
@@ -147,6 +149,14 @@ def sum_squares(g) -> float:
 
 def l2norm(g) -> float:
     return float(lib().gxo_l2norm(_p(g), g.size))
+
+
+def round_to_bf16(theta) -> np.ndarray:
+    """float64 array of float32 values -> uint16 bfloat16 patterns (round to nearest even)."""
+    theta = np.ascontiguousarray(theta, dtype=np.float64)
+    out = np.empty(theta.size, dtype=np.uint16)
+    lib().gxo_round_to_bf16(_p(theta), out.ctypes.data_as(ctypes.POINTER(ctypes.c_uint16)), theta.size)
+    return out
 
 
 def clip_coef(norm: float, max_norm: float) -> float:

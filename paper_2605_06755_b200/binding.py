@@ -68,6 +68,7 @@ _sigs = {
                                    ctypes.POINTER(_vp)]),
     "gxpo_destroy": (None, [_vp]),
     "gxpo_bind": (ctypes.c_int, [_vp, ctypes.POINTER(Tensor), ctypes.c_int]),
+    "gxpo_bind_model_weights": (ctypes.c_int, [_vp, ctypes.POINTER(_vp), ctypes.c_int, ctypes.c_int]),
     "gxpo_probe_step": (ctypes.c_int, [_vp, ctypes.c_int, _vp]),
     "gxpo_probe_step_deferred": (ctypes.c_int, [_vp, _vp]),
     "gxpo_extrapolate": (ctypes.c_int, [_vp, _vp]),
@@ -195,6 +196,15 @@ class Context:
 
     def bind(self, tensors: Sequence[TensorPtrs]):
         self._check(_lib.gxpo_bind(self._h, _pack(tensors), len(tensors)))
+
+    def bind_model_weights(self, ptrs, only_bf16_theta1: bool = False):
+        """ptrs: device pointers of the bfloat16 copies, one per bound tensor (0 = none),
+        or None to unbind."""
+        if ptrs is None:
+            self._check(_lib.gxpo_bind_model_weights(self._h, None, 0, 0))
+            return
+        arr = (_vp * max(1, len(ptrs)))(*[p or None for p in ptrs])
+        self._check(_lib.gxpo_bind_model_weights(self._h, arr, len(ptrs), 1 if only_bf16_theta1 else 0))
 
     def probe_step(self, which: int, stream=None):
         self._check(_lib.gxpo_probe_step(self._h, which, _stream_ptr(stream)))

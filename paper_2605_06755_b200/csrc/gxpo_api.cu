@@ -53,6 +53,8 @@ struct gxpo_ctx {
     long long num_chunks;
     int num_tensors;
     int bound;
+    std::vector<TensorDesc>* h_descs;  // host copy of the bound descriptors
+    int only_bf16_theta1;              // deferred first probe writes the bfloat16 copy only
     long long total_params;
     // reductions and gate
     double* d_partials;
@@ -174,6 +176,7 @@ StepParams make_step_params(gxpo_ctx* c, int which_grad, int in_sel, int out_sel
     p.snapshot = snapshot;
     p.want_norm = want_norm;
     p.write_state = 1;
+    p.emit = which_grad != 1;          // no backward pass is taken at theta^{t,2}
     p.gscale = c->gscale[which_grad];
     const gxpo_opt_cfg& o = c->opt;
     p.lr = (float)o.lr;
@@ -450,6 +453,7 @@ void gxpo_destroy(gxpo_ctx* c) {
     cudaFree(c->d_ring);
     cudaFree(c->d_result);
     if (c->h_result) cudaFreeHost(c->h_result);
+    delete c->h_descs;
     cudaFree(c->d_clip);
     cudaFree(c->d_gnorm);
     cudaFree(c->d_diag);
@@ -515,7 +519,35 @@ gxpo_status gxpo_bind(gxpo_ctx* c, const gxpo_tensor* list, int count) {
     c->total_params = total;
     c->gslow_aliased = aliased;
     c->diag_ready = 0;
+    c->only_bf16_theta1 = 0;
+    if (!c->h_descs) c->h_descs = new (std::nothrow) std::vector<TensorDesc>();
+    if (!c->h_descs) return fail(c, GXPO_ERR_INVALID_ARG, "out of host memory");
+    *c->h_descs = descs;
     c->bound = 1;
+    return GXPO_OK;
+}
+
+gxpo_status gxpo_bind_model_weights(gxpo_ctx* c, void* const* weights_bf16, int count, int only_bf16_theta1) {
+    if (!c) return GXPO_ERR_INVALID_ARG;
+    if (!c->bound || !c->h_descs) return fail(c, GXPO_ERR_STATE, "nothing bound: call gxpo_bind first");
+    if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "model weights can only be bound between steps");
+    std::vector<TensorDesc>& descs = *c->h_descs;
+    if (weights_bf16 && count != (int)descs.size())
+        return fail(c, GXPO_ERR_INVALID_ARG, "count %d does not match the %d bound tensors", count, (int)descs.size());
+    bool all = weights_bf16 != nullptr;
+    for (size_t i = 0; i < descs.size(); ++i) {
+        void* w = weights_bf16 ? weights_bf16[i] : nullptr;
+        if (((uintptr_t)w) & 1u) return fail(c, GXPO_ERR_ALIGNMENT, "tensor %d: bfloat16 pointer is not 2-byte aligned", (int)i);
+        if (!w && descs[i].n > 0) all = false;
+    }
+    if (only_bf16_theta1 && (!all || c->cfg.placement != GXPO_PLACE_PINGPONG))
+        return fail(c, GXPO_ERR_INVALID_ARG, "only_bf16_theta1 needs a bfloat16 buffer for every tensor and PINGPONG placement");
+    for (size_t i = 0; i < descs.size(); ++i)
+        descs[i].wb = static_cast<uint16_t*>(weights_bf16 ? weights_bf16[i] : nullptr);
+    CUDA_TRY(c, cudaDeviceSynchronize());
+    if (!descs.empty())
+        CUDA_TRY(c, cudaMemcpy(c->d_descs, descs.data(), descs.size() * sizeof(TensorDesc), cudaMemcpyHostToDevice));
+    c->only_bf16_theta1 = only_bf16_theta1 ? 1 : 0;
     return GXPO_OK;
 }
 
@@ -569,6 +601,7 @@ gxpo_status gxpo_probe_step_deferred(gxpo_ctx* c, void* stream) {
     StepParams p = (c->cfg.placement == GXPO_PLACE_PINGPONG) ? make_step_params(c, 0, 0, 1, 0, 0)
                                                              : make_step_params(c, 0, 0, 0, 1, 0);
     p.write_state = 0;
+    p.skip_out = c->only_bf16_theta1;
     gxpo_status st = launch_step(c, (cudaStream_t)stream, c->d_descs, c->d_chunks, c->num_chunks, none, p, c->d_sumsq);
     if (st != GXPO_OK) { c->t_opt -= 1; return st; }
     c->phase = PROBED0_DEFERRED;
@@ -851,6 +884,7 @@ gxpo_status gxpo_step_host(gxpo_ctx* c, const gxpo_tensor* list, int count, long
                 CUDA_TRY(c, cudaMemcpyAsync(st.g[k][2], static_cast<const char*>(T.g_slow) + off * gsz, len * gsz, cudaMemcpyHostToDevice, s));
             }
             TensorDesc d;
+            d.wb = nullptr;
             d.theta = st.theta[k]; d.work = st.work[k]; d.m = st.m[k]; d.v = st.v[k];
             d.g[0] = st.g[k][0]; d.g[1] = st.g[k][1]; d.g[2] = st.g[k][2];
             d.n = len;

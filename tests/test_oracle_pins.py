@@ -269,3 +269,24 @@ def test_clip_coefficient_matches_the_library_routine():
             np.testing.assert_allclose(p.grad.numpy(), g * c, rtol=1e-14, atol=0)
         assert (c == 1.0) == (max_norm / (norm + 1e-6) >= 1.0)
     assert ora.clip_coef(0.0, 1.0) == 1.0 and ora.clip_coef(2.0, 1.0) == pytest.approx(1 / (2 + 1e-6), rel=1e-15)
+
+
+def test_bf16_rounding_matches_the_library_conversion():
+    """Round-to-nearest-even float32 -> bfloat16 against torch's conversion, on random
+    values, exact ties, the largest finite values, subnormals, zeros and infinities."""
+    import torch
+    rng = np.random.default_rng(12)
+    x = np.concatenate([
+        rng.standard_normal(20000).astype(np.float32) * np.float32(0.02),
+        (rng.standard_normal(2000) * 1e30).astype(np.float32),
+        np.array([0.0, -0.0, np.inf, -np.inf, 3.4028235e38, -3.4028235e38, 1e-40, -1e-45, 1.0, -1.0], dtype=np.float32),
+        # exact ties: patterns ending in 0x8000 after an even and after an odd upper half
+        np.array([0x3F808000, 0x3F818000, 0xBF808000, 0x7F7F8000, 0x00008000, 0x00018000], dtype=np.uint32).view(np.float32),
+    ])
+    got = ora.round_to_bf16(x.astype(np.float64))
+    want = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    np.testing.assert_array_equal(got, want)
+    # ties go to even; the largest float32 rounds up to infinity
+    assert got[-6] == 0x3F80 and got[-5] == 0x3F82 and got[-3] == 0x7F80
+    nan = ora.round_to_bf16(np.array([np.nan]))
+    assert (nan[0] & 0x7F80) == 0x7F80 and (nan[0] & 0x007F) != 0
