@@ -402,3 +402,55 @@ def test_fused_call_order():
     ctx.slow_step()
     assert ctx.gate_update().t == 1
     ctx.close()
+
+
+@pytest.mark.parametrize("flow", ["deferred", "fused", "unfused", "fallback"])
+@pytest.mark.parametrize("placement", [0, 1])
+def test_no_sweep_writes_outside_its_tensors(flow, placement):
+    """Every output buffer (theta, work, m, v and the bfloat16 copies) sits between two
+    guard bands filled with a sentinel; after a step the bands must be untouched and the
+    read-only gradient buffers bit-identical.  Sizes end mid-vector, mid-tile and
+    mid-chunk, aligned and misaligned."""
+    import torch
+    b = _binding()
+    sizes = [1, 7, 2049, 32768 + 3, 2 * 32768 - 1, 70001]
+    offsets = [0, 3, 0, 0, 1, 0]
+    GUARD = 4096
+    sentinel = 1234.5
+
+    def guarded(x):
+        big = torch.full((x.numel() + 2 * GUARD,), sentinel, dtype=x.dtype, device="cuda")
+        big[GUARD:GUARD + x.numel()] = x
+        return big, big[GUARD:GUARD + x.numel()]
+
+    bigs, ptrs, grads, wptrs = [], [], [], []
+    for i, (n, off) in enumerate(zip(sizes, offsets)):
+        pr = _problem(n, seed=500 + i, grad_dtype="bf16", zero_frac=0.03, offset=off)
+        views = []
+        for t in (pr.theta, pr.work, pr.m, pr.v):
+            big, view = guarded(t if off == 0 else torch.cat([t.new_zeros(off), t]))
+            bigs.append(big)
+            views.append(view[off:] if off else view)
+        wbig, wview = guarded(torch.zeros(n + off, dtype=torch.bfloat16, device="cuda"))
+        bigs.append(wbig)
+        wptrs.append((wview[off:] if off else wview).data_ptr())
+        ptrs.append(b.tensor_ptrs(views[0], views[1], views[2], views[3], pr.g0, pr.g1, pr.gs))
+        grads.append((pr, [pr.g0.clone(), pr.g1.clone(), pr.gs.clone()]))
+    ctx, cfg, opt = _ctx(b, "bf16", lr=1e-3, K=5, alpha=0.5, placement=placement)
+    ctx.bind(ptrs)
+    ctx.bind_model_weights(wptrs)
+    ctx.enable_diagnostics(True)
+    for _ in range(2):
+        if flow == "fallback":
+            ctx.probe_step(-1)
+        else:
+            ctx.active_step(allow_nonfinite=True, fused=(flow == "fused"), deferred=(flow == "deferred"))
+    torch.cuda.synchronize()
+    for big in bigs:
+        s = torch.tensor(sentinel, dtype=big.dtype, device="cuda")
+        assert torch.all(big[:GUARD] == s) and torch.all(big[-GUARD:] == s)
+    for pr, (g0, g1, gs) in grads:
+        assert torch.equal(pr.g0.view(torch.int16), g0.view(torch.int16))
+        assert torch.equal(pr.g1.view(torch.int16), g1.view(torch.int16))
+        assert torch.equal(pr.gs.view(torch.int16), gs.view(torch.int16))
+    ctx.close()
