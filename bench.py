@@ -49,7 +49,7 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="qwen25_7b",
-                    choices=["qwen25_7b", "llama31_8b", "flat_1p54b", "lora_qwen25_7b", "small", "flat"])
+                    choices=["qwen25_7b", "llama31_8b", "flat_1p54b", "flat_2p5b", "lora_qwen25_7b", "small", "flat"])
     ap.add_argument("--params", type=int, default=1 << 26, help="size of the 'flat' workload")
     ap.add_argument("--layers", type=int, default=0, help="override the decoder depth (0 = full)")
     ap.add_argument("--K", type=int, default=5)
@@ -83,6 +83,8 @@ def workload_shapes(args):
         return w.lora_qwen25_7b_shapes(), "rank-128 LoRA adapters (q, k, v, o) of a Qwen2.5-7B-shaped decoder"
     if args.workload == "flat":
         return [("flat", args.params)], f"flat {args.params}-parameter buffer"
+    if args.workload == "flat_2p5b":
+        return [("flat", 2_500_000_007)], "flat 2,500,000,007-parameter buffer (offsets beyond 2^31 elements)"
     if args.workload == "flat_1p54b":
         return [("flat", w.FLAT_QWEN25_1P5B)], "flat 1.54e9-parameter buffer"
     return w.qwen25_7b_shapes(args.layers or 1), "Qwen2.5-7B-shaped list, reduced depth"

@@ -45,7 +45,9 @@ typedef enum {
     GXPO_ERR_ALIGNMENT = 2,   /* a pointer is not aligned to its element size */
     GXPO_ERR_STATE = 3,       /* call out of order for Algorithm 1, or nothing bound */
     GXPO_ERR_CUDA = 4,        /* a CUDA runtime call failed; see gxpo_last_error */
-    GXPO_ERR_TIMEOUT = 5,     /* a bounded device-side wait gave up */
+    GXPO_ERR_TIMEOUT = 5,     /* reserved for a bounded device-side wait that gave up; no kernel
+                                 here waits on another (the reductions are wait-free), so it
+                                 is not returned today */
     GXPO_ERR_NONFINITE = 6    /* ||g_slow|| was not finite; the gate was tripped */
 } gxpo_status;
 

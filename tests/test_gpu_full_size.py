@@ -97,12 +97,12 @@ def _check_window(keep, lo, hi, st, scale, theta0, theta2, alpha, what, rtol=2e-
     return nsat
 
 
-def _one_active_step_vs_oracle(workload, lr, picks_fn, full_oracle_norm):
+def _one_active_step_vs_oracle(workload, lr, picks_fn, full_oracle_norm, extra_windows=()):
     import torch
     b, ctx, cfg, opt, shapes, desc, alias, d, keep = _setup(workload, lr)
     assert "reduced" not in desc, desc           # the full size is the point of this test
     gcfg, ocfg = gu.ora_cfgs(cfg, opt)
-    wins = _windows(shapes, picks_fn(shapes))
+    wins = _windows(shapes, picks_fn(shapes)) + list(extra_windows)
     before = [_grab(keep, lo, hi) for lo, hi in wins]
     gs = keep[6]
     if full_oracle_norm:
@@ -142,6 +142,16 @@ def test_flat_1p54b_one_active_step(lr):
     def picks(shapes):
         return [(0, "head"), (0, "chunk"), (0, "mid"), (0, "tail")]
     _one_active_step_vs_oracle("flat_1p54b", lr, picks, full_oracle_norm=True)
+
+
+def test_flat_2p5b_offsets_beyond_two_to_the_31():
+    """One tensor of 2,500,000,007 parameters (odd length): element offsets pass 2^31 and
+    byte offsets pass 2^32 and 2^33; windows sit on those boundaries and at the ragged end."""
+    def picks(shapes):
+        return [(0, "head"), (0, "tail")]
+    extra = [(2 ** 31 - WIN // 2, 2 ** 31 + WIN // 2), (2 ** 30 - WIN // 2, 2 ** 30 + WIN // 2),
+             (2 ** 31 + 2 ** 28 - 777, 2 ** 31 + 2 ** 28 + WIN)]
+    _one_active_step_vs_oracle("flat_2p5b", 1e-3, picks, full_oracle_norm=False, extra_windows=extra)
 
 
 def _decoder_picks(shapes):
