@@ -19,7 +19,10 @@
  *   optim_step_gd + extrapolate : closed form of Corollary 1 / Appendix A.6 on a
  *                                 diagonal quadratic, brute-force K explicit steps
  *   scale factor                : identities of Eq. (scale_factor), Eq. (geom_sum_def)
- *   optim_step_adamw            : one library AdamW step in float64, three in a row
+ *   optim_step_adamw            : one library AdamW step in float64, three in a row; whole
+ *                                 active steps against the library optimizer with a
+ *                                 hand-written closed-form reposition
+ *   bf16 rounding, clip coef    : the library conversion / clipping routine
  *   l2norm                      : closed forms, a library norm
  *   gate                        : hand-built norm streams, a library mean/std,
  *                                 printed (shutoff step, total backward passes) rows

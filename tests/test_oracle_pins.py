@@ -225,6 +225,45 @@ def test_active_step_advances_optimizer_state_three_times():
     np.testing.assert_allclose(st.v, v, rtol=1e-13)
 
 
+def test_adamw_active_steps_against_library_optimizer_with_manual_reposition():
+    """Algorithm 1's active branch with the library's AdamW as OptimStep: two fast steps,
+    the parameters repositioned by hand with the closed form (1 - r^K) / (1 - r^2) of
+    Eq. (scale_factor), the third step with g_slow; optimizer state never rewound.  Two
+    consecutive active steps, float64."""
+    import torch
+    rng = np.random.default_rng(21)
+    n, K, alpha, delta = 200, 5, 0.5, 1e-8
+    theta0 = rng.standard_normal(n)
+    opt = ora.OptCfg(kind="adamw", lr=1e-2, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    st = ora.State(theta0, opt)
+    p = torch.nn.Parameter(torch.from_numpy(theta0.copy()))
+    lib = torch.optim.AdamW([p], lr=1e-2, betas=(0.9, 0.999), eps=1e-8, weight_decay=0.01)
+    for step in range(2):
+        g0 = rng.standard_normal(n)
+        g0[::17] = 0.0                                  # some inactive coordinates
+        g1 = g0 * rng.uniform(0.3, 1.3, n) + (g0 == 0) * 0.5
+        gs = rng.standard_normal(n)
+        grads = [g0, g1, gs]
+        nrm = ora.active_step(st, ora.GxpoCfg(K=K, alpha=alpha, delta=delta), lambda w, th: grads[w])
+        start = p.detach().numpy().copy()
+        for g in (g0, g1):
+            p.grad = torch.from_numpy(g.copy())
+            lib.step()
+        th2 = p.detach().numpy().copy()
+        act = np.abs(g0) > delta
+        r = np.where(act, g1 / np.where(act, g0, 1.0), 0.0)
+        scale = np.where(act, (1 - r ** K) / (1 - r ** 2), 1.0)
+        with torch.no_grad():
+            p.copy_(torch.from_numpy(start + alpha * (th2 - start) * scale))
+        p.grad = torch.from_numpy(gs.copy())
+        lib.step()
+        np.testing.assert_allclose(st.theta, p.detach().numpy(), rtol=1e-10, atol=1e-12)
+        np.testing.assert_allclose(st.m, lib.state[p]["exp_avg"].numpy(), rtol=1e-12, atol=1e-15)
+        np.testing.assert_allclose(st.v, lib.state[p]["exp_avg_sq"].numpy(), rtol=1e-12, atol=1e-18)
+        assert nrm == pytest.approx(np.linalg.norm(gs), rel=1e-14)
+    assert st.t_opt == 6 and int(lib.state[p]["step"]) == 6
+
+
 # ---------------------------------------------------------------------------
 # norm
 # ---------------------------------------------------------------------------
