@@ -49,7 +49,7 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="qwen25_7b",
-                    choices=["qwen25_7b", "llama31_8b", "flat_1p54b", "flat_2p5b", "lora_qwen25_7b", "small", "flat"])
+                    choices=["qwen25_7b", "llama31_8b", "flat_1p54b", "flat_2p5b", "lora_qwen25_7b", "surrogate_1e8", "small", "flat"])
     ap.add_argument("--params", type=int, default=1 << 26, help="size of the 'flat' workload")
     ap.add_argument("--layers", type=int, default=0, help="override the decoder depth (0 = full)")
     ap.add_argument("--K", type=int, default=5)
@@ -480,10 +480,89 @@ def run_e2e(torch, b, args, cfg, opt):
                       f"streamed through gxpo_step_host in 8388608-parameter pieces"}
 
 
+def run_surrogate(args):
+    """The diagonal-quadratic surrogate at n = 1e8 (plain GD, eta = 0.1, gradients computed
+    in-kernel): `--steps` consecutive active steps, once through the fused harness kernel
+    (16 B/param) and once through the library calls with the harness gradient kernel standing
+    in for the backward passes (3 x 16 + 12 + 12 + 20 + 12 = 104 B/param, fp32 gradients)."""
+    import torch
+
+    from paper_2605_06755_b200 import build
+    build.build_library()
+    from paper_2605_06755_b200 import binding as b
+    from paper_2605_06755_b200 import workloads as w
+    torch.cuda.set_device(0)
+    n, eta = 100_000_000, 0.1
+    a_np, b_np, t0_np = w.quadratic_surrogate(n, 0)
+    a, bb, t0 = (torch.from_numpy(x).cuda() for x in (a_np, b_np, t0_np))
+    peak, peak_kind = measured_peak_gbs()
+    stream = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # fused harness kernel
+    theta = t0.clone()
+    scratch = torch.zeros(b.quad_scratch_bytes(), dtype=torch.uint8, device="cuda")
+    sumsq = torch.zeros(1, dtype=torch.float64, device="cuda")
+    def fused_step():
+        b.quad_active_step(theta.data_ptr(), a.data_ptr(), bb.data_ptr(), n, eta, args.K, 1.0, 1e-8, 0.0,
+                           sumsq.data_ptr(), scratch.data_ptr(), stream)
+    for _ in range(max(args.warmup, 3)):
+        fused_step()
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(args.steps):
+        fused_step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms_fused = e0.elapsed_time(e1) / args.steps
+    # the library calls
+    theta2, work = t0.clone(), torch.empty_like(t0)
+    g0, g1, gs = (torch.empty_like(t0) for _ in range(3))
+    cfg, opt = b.make_cfg(kind=b.OPT_GD, lr=eta, K=args.K, alpha=1.0, delta=1e-8)
+    ctx = b.Context(cfg, opt, b.F32)
+    ctx.bind([b.tensor_ptrs(theta2, work, None, None, g0, g1, gs)])
+    def api_step():
+        b.quad_grad(theta2.data_ptr(), a.data_ptr(), bb.data_ptr(), g0.data_ptr(), n, stream)
+        ctx.probe_step(0, stream)
+        b.quad_grad(work.data_ptr(), a.data_ptr(), bb.data_ptr(), g1.data_ptr(), n, stream)
+        ctx.probe_step(1, stream)
+        ctx.extrapolate(stream)
+        b.quad_grad(theta2.data_ptr(), a.data_ptr(), bb.data_ptr(), gs.data_ptr(), n, stream)
+        ctx.slow_step(stream)
+        return ctx.gate_update(stream)
+    for _ in range(max(args.warmup, 3)):
+        api_step()
+    torch.cuda.synchronize()
+    l0 = ctx.launch_count()
+    e0.record(stream)
+    for _ in range(args.steps):
+        res = api_step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms_api = e0.elapsed_time(e1) / args.steps
+    launches = ctx.launch_count() - l0 + 3 * args.steps
+    gbs = 16 * n / (ms_fused * 1e-3) / 1e9
+    line = {"metric": METRIC, "value": n / (ms_fused * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_fused, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "diagonal-quadratic surrogate, n = 1e8, plain GD eta = 0.1, gradients in-kernel",
+                       "K": args.K, "alpha": 1.0, "step": "fused harness kernel (16 B/param)",
+                       "l2": "inputs larger than L2 (no flush needed)"},
+            "roofline": {"bound": "hbm", "kernel": "quad_active_kernel", "achieved": gbs, "peak": peak, "unit": "GB/s",
+                         "frac": gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                         "algorithmic_bytes_per_launch": 16 * n},
+            "library_calls": {"ms_per_step": ms_api, "bytes_per_param": 104,
+                              "gbs": 104 * n / (ms_api * 1e-3) / 1e9, "gate_norm": res.norm},
+            "gpu_launches": launches + args.steps}
+    ctx.close()
+    print(json.dumps(line), flush=True)
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "surrogate_1e8":
+        run_surrogate(args)
     else:
         run_ours(args)
 
