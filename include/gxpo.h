@@ -25,6 +25,9 @@
  *   - Vector (128/256-bit) access is used for a tensor when all of its bound
  *     pointers are 32-byte aligned; otherwise that tensor takes a slower scalar
  *     path with identical results.  Any n >= 0 is accepted; n == 0 is a no-op.
+ *   - The calls of one context share its small device scratch (partial sums, counters):
+ *     issue them on one stream, or order the streams yourself, so that no two of its
+ *     kernels run at the same time.
  *   - A context is not thread-safe; use one per host thread or lock around it.
  *   - One GPU per context: the device current at gxpo_create.
  */

@@ -27,3 +27,12 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_sessionstart(session):
+    """Build the CUDA library and the oracle when they are missing or older than their
+    sources (both are build products and not in the repository's history)."""
+    from oracle import gxpo_oracle
+    from paper_2605_06755_b200 import build
+    build.build_library()
+    gxpo_oracle.build()
