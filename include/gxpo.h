@@ -210,6 +210,20 @@ gxpo_status gxpo_slow_step(gxpo_ctx* ctx, void* stream);
  * norm is Inf/NaN -- that rule is this library's, not the paper's. */
 gxpo_status gxpo_gate_update(gxpo_ctx* ctx, void* stream, gxpo_gate_result* out);
 
+/* The same update without the wait: the gate kernel and its 64-byte read-back are only
+ * enqueued on `stream`, and the call returns at once, so the host can go on issuing work
+ * (the next rollouts, the next backward pass) while the step drains.  The outcome is
+ * collected by whichever call needs it first: gxpo_gate_last, gxpo_gate_peek, the next
+ * gxpo_probe_step(ctx, 0) / gxpo_probe_step_deferred (they must know whether the gate
+ * has tripped), gxpo_backward_passes, gxpo_state_export -- each waits for the read-back
+ * if it is still in flight.  state: SLOW_DONE -> IDLE. */
+gxpo_status gxpo_gate_update_async(gxpo_ctx* ctx, void* stream);
+
+/* Outcome of the most recent gate update (waits for it if it is still in flight).
+ * Returns NONFINITE, like gxpo_gate_update, when that update saw a non-finite norm;
+ * STATE when no update has run yet.  `out` may be NULL. */
+gxpo_status gxpo_gate_last(gxpo_ctx* ctx, gxpo_gate_result* out);
+
 /* Sharded parameter sets (one process per GPU, each holding a slice of every
  * tensor or a subset of the list): the only cross-shard quantity of the whole
  * update is sum(g_slow^2).  Point the context at a caller-owned DEVICE double;
@@ -271,7 +285,8 @@ gxpo_status gxpo_enable_diagnostics(gxpo_ctx* ctx, int on);
  * `stream` (one small read-back).  Errors: STATE otherwise. */
 gxpo_status gxpo_get_diagnostics(gxpo_ctx* ctx, void* stream, gxpo_diagnostics* out);
 
-/* Host-side view of the gate, no device work. */
+/* Host-side view of the gate; no device work (it only waits if a gxpo_gate_update_async
+ * read-back is still in flight). */
 gxpo_status gxpo_gate_peek(const gxpo_ctx* ctx, int* active, long long* s_star, long long* t);
 
 /* Optimizer step count so far (3 per active step, 1 per fallback step). */

@@ -75,6 +75,8 @@ _sigs = {
     "gxpo_probe_extrapolate": (ctypes.c_int, [_vp, _vp]),
     "gxpo_slow_step": (ctypes.c_int, [_vp, _vp]),
     "gxpo_gate_update": (ctypes.c_int, [_vp, _vp, ctypes.POINTER(GateResult)]),
+    "gxpo_gate_update_async": (ctypes.c_int, [_vp, _vp]),
+    "gxpo_gate_last": (ctypes.c_int, [_vp, ctypes.POINTER(GateResult)]),
     "gxpo_set_sumsq_buffer": (ctypes.c_int, [_vp, _vp]),
     "gxpo_set_grad_scale": (ctypes.c_int, [_vp, ctypes.c_int, _vp]),
     "gxpo_clip_grad_norm": (ctypes.c_int, [_vp, ctypes.c_int, ctypes.c_double, _vp]),
@@ -224,6 +226,17 @@ class Context:
     def gate_update(self, stream=None, allow_nonfinite: bool = False) -> GateResult:
         res = GateResult()
         st = _lib.gxpo_gate_update(self._h, _stream_ptr(stream), ctypes.byref(res))
+        if st == ERR_NONFINITE and allow_nonfinite:
+            return res
+        self._check(st)
+        return res
+
+    def gate_update_async(self, stream=None):
+        self._check(_lib.gxpo_gate_update_async(self._h, _stream_ptr(stream)))
+
+    def gate_last(self, allow_nonfinite: bool = False) -> GateResult:
+        res = GateResult()
+        st = _lib.gxpo_gate_last(self._h, ctypes.byref(res))
         if st == ERR_NONFINITE and allow_nonfinite:
             return res
         self._check(st)

@@ -65,6 +65,10 @@ struct gxpo_ctx {
     double* d_ring;
     GateResult* d_result;
     GateResult* h_result;              // pinned
+    cudaEvent_t gate_done;             // recorded after the gate's read-back
+    int gate_pending;                  // a read-back is in flight (gxpo_gate_update_async)
+    int have_gate;
+    gxpo_gate_result last_gate;
     // per-step diagnostics (off by default)
     // gradient scaling: per gradient a device scalar (caller's, or clip[] below), or null
     const float* gscale[3];            // what the sweeps use
@@ -302,29 +306,46 @@ void expire_clips(gxpo_ctx* c) {
     for (int k = 0; k < 3; ++k) c->gscale[k] = c->user_gscale[k];
 }
 
-gxpo_status run_gate(gxpo_ctx* c, cudaStream_t s, const double* sumsq, gxpo_gate_result* out) {
+// Enqueue the gate kernel and its read-back; the host learns the outcome in finish_gate.
+// t advances by one whatever the outcome, so the host mirror moves on at once.
+gxpo_status launch_gate(gxpo_ctx* c, cudaStream_t s, const double* sumsq) {
     gate_kernel<<<1, 32, 0, s>>>(c->d_gate, c->d_ring, sumsq, c->t, c->cfg.tau, c->cfg.gate_eps,
                                  c->cfg.window, c->cfg.min_history, c->cfg.std_ddof, c->d_result);
     c->launches += 1;
     CUDA_TRY(c, cudaGetLastError());
     CUDA_TRY(c, cudaMemcpyAsync(c->h_result, c->d_result, sizeof(GateResult), cudaMemcpyDeviceToHost, s));
-    CUDA_TRY(c, cudaStreamSynchronize(s));
-    const GateResult r = *c->h_result;
-    c->t = r.t;
-    c->s_star = r.s_star;
-    if (out) {
-        out->active = r.active;
-        out->tripped = r.tripped;
-        out->t = r.t;
-        out->s_star = r.s_star;
-        out->norm = r.norm;
-        out->z = r.z;
-        out->mu = r.mu;
-        out->sigma = r.sigma;
-    }
-    if (!std::isfinite(r.norm))
-        return fail(c, GXPO_ERR_NONFINITE, "||g_slow|| is not finite at step %lld; gate tripped", r.t - 1);
+    CUDA_TRY(c, cudaEventRecord(c->gate_done, s));
+    c->gate_pending = 1;
+    c->t += 1;
     return GXPO_OK;
+}
+
+// Wait for a pending gate read-back (if any) and fold it into the host mirror.
+gxpo_status finish_gate(gxpo_ctx* c) {
+    if (!c->gate_pending) return GXPO_OK;
+    CUDA_TRY(c, cudaEventSynchronize(c->gate_done));
+    c->gate_pending = 0;
+    const GateResult r = *c->h_result;
+    c->s_star = r.s_star;
+    gxpo_gate_result& o = c->last_gate;
+    o.active = r.active; o.tripped = r.tripped; o.t = r.t; o.s_star = r.s_star;
+    o.norm = r.norm; o.z = r.z; o.mu = r.mu; o.sigma = r.sigma;
+    c->have_gate = 1;
+    return GXPO_OK;
+}
+
+gxpo_status gate_outcome(gxpo_ctx* c, gxpo_gate_result* out) {
+    if (out) *out = c->last_gate;
+    if (!std::isfinite(c->last_gate.norm))
+        return fail(c, GXPO_ERR_NONFINITE, "||g_slow|| is not finite at step %lld; gate tripped", c->last_gate.t - 1);
+    return GXPO_OK;
+}
+
+gxpo_status run_gate(gxpo_ctx* c, cudaStream_t s, const double* sumsq, gxpo_gate_result* out) {
+    gxpo_status st = launch_gate(c, s, sumsq);
+    if (st == GXPO_OK) st = finish_gate(c);
+    if (st != GXPO_OK) return st;
+    return gate_outcome(c, out);
 }
 
 void free_staging(gxpo_ctx* c) {
@@ -418,6 +439,7 @@ gxpo_status gxpo_create(const gxpo_cfg* cfg, const gxpo_opt_cfg* opt, int grad_d
     if (e == cudaSuccess) e = cudaMalloc(&c->d_ring, (size_t)cfg->window * sizeof(double));
     if (e == cudaSuccess) e = cudaMalloc(&c->d_result, sizeof(GateResult));
     if (e == cudaSuccess) e = cudaMallocHost(&c->h_result, sizeof(GateResult));
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->gate_done, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaMalloc(&c->d_clip, 3 * sizeof(float));
     if (e == cudaSuccess) e = cudaMalloc(&c->d_gnorm, 6 * sizeof(double));
     if (e == cudaSuccess) e = cudaMalloc(&c->d_diag, (kDiagN + 1) * sizeof(double));
@@ -453,6 +475,7 @@ void gxpo_destroy(gxpo_ctx* c) {
     cudaFree(c->d_ring);
     cudaFree(c->d_result);
     if (c->h_result) cudaFreeHost(c->h_result);
+    if (c->gate_done) cudaEventDestroy(c->gate_done);
     delete c->h_descs;
     cudaFree(c->d_clip);
     cudaFree(c->d_gnorm);
@@ -570,6 +593,7 @@ gxpo_status gxpo_probe_step(gxpo_ctx* c, int which, void* stream) {
     }
     if (which == 0) {
         if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "probe step 0 must start a step");
+        { gxpo_status fg = finish_gate(c); if (fg != GXPO_OK) return fg; }
         if (!gate_active(c)) return fail(c, GXPO_ERR_STATE, "gate has tripped (s*=%lld, t=%lld): only fallback steps are legal", c->s_star, c->t);
         c->t_opt += 1;
         StepParams p = (place == GXPO_PLACE_PINGPONG) ? make_step_params(c, 0, 0, 1, 0, 0)
@@ -595,6 +619,7 @@ gxpo_status gxpo_probe_step_deferred(gxpo_ctx* c, void* stream) {
     if (!c) return GXPO_ERR_INVALID_ARG;
     if (!c->bound) return fail(c, GXPO_ERR_STATE, "nothing bound: call gxpo_bind first");
     if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "probe step 0 must start a step");
+    { gxpo_status fg = finish_gate(c); if (fg != GXPO_OK) return fg; }
     if (!gate_active(c)) return fail(c, GXPO_ERR_STATE, "gate has tripped (s*=%lld, t=%lld): only fallback steps are legal", c->s_star, c->t);
     const TensorDesc none = {};
     c->t_opt += 1;
@@ -667,6 +692,25 @@ gxpo_status gxpo_gate_update(gxpo_ctx* c, void* stream, gxpo_gate_result* out) {
     c->diag_ready = c->diag_on;
     expire_clips(c);
     return run_gate(c, (cudaStream_t)stream, c->user_sumsq ? c->user_sumsq : c->d_sumsq, out);
+}
+
+gxpo_status gxpo_gate_update_async(gxpo_ctx* c, void* stream) {
+    if (!c) return GXPO_ERR_INVALID_ARG;
+    if (c->phase != SLOW_DONE) return fail(c, GXPO_ERR_STATE, "gate update must follow the slow step");
+    gxpo_status st = finish_gate(c);
+    if (st != GXPO_OK) return st;
+    c->phase = IDLE;
+    c->diag_ready = c->diag_on;
+    expire_clips(c);
+    return launch_gate(c, (cudaStream_t)stream, c->user_sumsq ? c->user_sumsq : c->d_sumsq);
+}
+
+gxpo_status gxpo_gate_last(gxpo_ctx* c, gxpo_gate_result* out) {
+    if (!c) return GXPO_ERR_INVALID_ARG;
+    gxpo_status st = finish_gate(c);
+    if (st != GXPO_OK) return st;
+    if (!c->have_gate) return fail(c, GXPO_ERR_STATE, "no gate update has run yet");
+    return gate_outcome(c, out);
 }
 
 gxpo_status gxpo_set_sumsq_buffer(gxpo_ctx* c, double* sumsq_dev) {
@@ -746,6 +790,7 @@ gxpo_status gxpo_get_diagnostics(gxpo_ctx* c, void* stream, gxpo_diagnostics* ou
 
 gxpo_status gxpo_gate_peek(const gxpo_ctx* c, int* active, long long* s_star, long long* t) {
     if (!c) return GXPO_ERR_INVALID_ARG;
+    { gxpo_status fg = finish_gate(const_cast<gxpo_ctx*>(c)); if (fg != GXPO_OK) return fg; }
     if (active) *active = gate_active(c) ? 1 : 0;
     if (s_star) *s_star = c->s_star;
     if (t) *t = c->t;
@@ -756,6 +801,7 @@ long long gxpo_optimizer_steps(const gxpo_ctx* c) { return c ? c->t_opt : -1; }
 
 long long gxpo_backward_passes(const gxpo_ctx* c) {
     if (!c) return -1;
+    if (finish_gate(const_cast<gxpo_ctx*>(c)) != GXPO_OK) return -1;
     const long long s = (c->s_star < 0 || c->s_star > c->t) ? c->t : c->s_star;
     return 3 * s + (c->t - s);
 }
@@ -808,6 +854,7 @@ gxpo_status gxpo_state_export(gxpo_ctx* c, void* buf, size_t* len) {
     if (!buf) { *len = need; return GXPO_OK; }
     if (*len < need) { *len = need; return fail(c, GXPO_ERR_INVALID_ARG, "buffer too small: need %zu bytes", need); }
     if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "state export in the middle of a step");
+    { gxpo_status fg = finish_gate(c); if (fg != GXPO_OK) return fg; }
     CUDA_TRY(c, cudaDeviceSynchronize());
     GateState g;
     CUDA_TRY(c, cudaMemcpy(&g, c->d_gate, sizeof(g), cudaMemcpyDeviceToHost));
@@ -826,6 +873,7 @@ gxpo_status gxpo_state_import(gxpo_ctx* c, const void* buf, size_t len) {
     const size_t need = sizeof(StateHeader) + (size_t)c->cfg.window * sizeof(double);
     if (len < need) return fail(c, GXPO_ERR_INVALID_ARG, "state blob too short");
     if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "state import in the middle of a step");
+    { gxpo_status fg = finish_gate(c); if (fg != GXPO_OK) return fg; }
     StateHeader h;
     std::memcpy(&h, buf, sizeof(h));
     if (h.magic != kMagic || h.version != 1) return fail(c, GXPO_ERR_INVALID_ARG, "not a GXPO state blob");
@@ -847,6 +895,7 @@ gxpo_status gxpo_step_host(gxpo_ctx* c, const gxpo_tensor* list, int count, long
     if (!c) return GXPO_ERR_INVALID_ARG;
     if (count < 0 || (count > 0 && !list)) return fail(c, GXPO_ERR_INVALID_ARG, "bad list/count");
     if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "host step in the middle of a device step");
+    { gxpo_status fg = finish_gate(c); if (fg != GXPO_OK) return fg; }
     if (staging_elems <= 0) staging_elems = 1LL << 24;
     staging_elems = (staging_elems + kChunk - 1) / kChunk * kChunk;
     for (int i = 0; i < count; ++i) {

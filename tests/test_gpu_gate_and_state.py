@@ -254,3 +254,52 @@ def test_state_export_import_round_trip():
         bctx.state_import(b"\0" * len(blob))
     for c in (ref, a, bctx):
         c.close()
+
+
+def test_async_gate_update_gives_the_same_decisions():
+    """gxpo_gate_update_async + whoever collects the outcome (the next probe step, gate_peek,
+    gate_last) against the synchronous call, on a stream that trips at step 9."""
+    import torch
+    b = _binding()
+    rng = np.random.default_rng(3)
+    norms = np.abs(1.0 + 0.01 * rng.standard_normal(14)).astype(np.float32)
+    norms[9] = 2.0
+
+    def make():
+        cfg, opt = b.make_cfg(kind=b.OPT_GD, lr=0.0, tau=3.0, window=8)
+        ctx = b.Context(cfg, opt, b.F32)
+        th = torch.zeros(1, device="cuda"); wk = torch.zeros(1, device="cuda")
+        g = torch.ones(1, device="cuda"); gs = torch.zeros(1, device="cuda")
+        ctx.bind([b.tensor_ptrs(th, wk, None, None, g, g, gs)])
+        return ctx, gs, (th, wk, g)
+
+    sync, gs_s, k1 = make()
+    asyn, gs_a, k2 = make()
+    with pytest.raises(b.GxpoError) as e:
+        asyn.gate_last()
+    assert e.value.status == b.ERR_STATE
+    for t, x in enumerate(norms):
+        assert sync.gate_peek() == asyn.gate_peek()
+        if not sync.gate_peek()[0]:
+            sync.probe_step(-1); asyn.probe_step(-1)
+            continue
+        gs_s.fill_(float(x)); gs_a.fill_(float(x))
+        want = sync.active_step()
+        asyn.probe_step_deferred(); asyn.probe_extrapolate(); asyn.slow_step()
+        asyn.gate_update_async()
+        if t % 3 == 0:
+            got = asyn.gate_last()                       # collected explicitly
+        elif t % 3 == 1:
+            asyn.gate_peek(); got = asyn.gate_last()     # collected by gate_peek
+        else:
+            got = None                                   # collected by the next probe step
+        if got is not None:
+            assert (got.tripped, got.s_star, got.t, got.active) == (want.tripped, want.s_star, want.t, want.active)
+            assert got.norm == want.norm and (got.z == want.z or (math.isnan(got.z) and math.isnan(want.z)))
+    assert sync.gate_peek() == asyn.gate_peek() and sync.gate_peek()[1] == 10
+    assert sync.backward_passes() == asyn.backward_passes() == 3 * 10 + 4
+    assert asyn.state_export() == sync.state_export()
+    with pytest.raises(b.GxpoError) as e:
+        asyn.probe_step_deferred()                       # tripped: the active phase is over
+    assert e.value.status == b.ERR_STATE
+    sync.close(); asyn.close()
