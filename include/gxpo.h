@@ -48,9 +48,10 @@ typedef enum {
     GXPO_ERR_ALIGNMENT = 2,   /* a pointer is not aligned to its element size */
     GXPO_ERR_STATE = 3,       /* call out of order for Algorithm 1, or nothing bound */
     GXPO_ERR_CUDA = 4,        /* a CUDA runtime call failed; see gxpo_last_error */
-    GXPO_ERR_TIMEOUT = 5,     /* reserved for a bounded device-side wait that gave up; no kernel
-                                 here waits on another (the reductions are wait-free), so it
-                                 is not returned today */
+    GXPO_ERR_TIMEOUT = 5,     /* a bounded device-side wait gave up (only the bulk-copy staged
+                                 variant of the fused sweep waits on anything; the default
+                                 kernels and all reductions are wait-free); reported by the
+                                 gate update that ends the step */
     GXPO_ERR_NONFINITE = 6    /* ||g_slow|| was not finite; the gate was tripped */
 } gxpo_status;
 
@@ -315,7 +316,10 @@ gxpo_status gxpo_step_host(gxpo_ctx* ctx, const gxpo_tensor* list, int count,
                            long long staging_elems, void* stream, gxpo_gate_result* out);
 
 /* Launch-shape knobs, for benchmarking: resident CTAs per SM (0 = default), the
- * memory-access variant (0 = default, 1 = 128-bit loads, 2 = 256-bit loads) and the
+ * memory-access variant (0 = default, 1 = 128-bit loads, 2 = 256-bit loads, 3 = 256-bit
+ * loads plus, for gxpo_probe_extrapolate, a producer thread that stages whole tiles in
+ * shared memory with bulk asynchronous copies -- measured slower than 2, kept for
+ * comparison) and the
  * number of 2048-element tiles a CTA takes per round-robin turn (0 = default: 16, or
  * 8 / 4 for lists of only a few thousand 32768-element chunks; else 1, 2, 4, 8 or 16).  Element-wise results are identical across all settings; only the
  * summation order of the norm changes. */
@@ -361,6 +365,13 @@ gxpo_status gxpo_slow_step_noalloc(float* theta, float* m, float* v, const void*
                                    long long n, int grad_dtype, const gxpo_opt_cfg* opt,
                                    long long t_opt, double* sumsq_dev, void* stream,
                                    char* errbuf, size_t errbuf_len);
+
+/* Exercises the bounded wait of the bulk-copy variant end to end: a one-thread kernel waits
+ * on a barrier that nothing completes, gives up after a few thousand polls and raises the
+ * device error word, which this call reads back and clears.  Returns GXPO_ERR_TIMEOUT when
+ * that happened -- the expected outcome -- and GXPO_OK otherwise.  The context stays
+ * usable.  Only legal between steps; waits for `stream`. */
+gxpo_status gxpo_selftest_bounded_wait(gxpo_ctx* ctx, void* stream);
 
 /* Number of kernels this context has launched so far. */
 long long gxpo_launch_count(const gxpo_ctx* ctx);

@@ -92,6 +92,7 @@ _sigs = {
     "gxpo_step_host": (ctypes.c_int, [_vp, ctypes.POINTER(Tensor), ctypes.c_int,
                                       ctypes.c_longlong, _vp, ctypes.POINTER(GateResult)]),
     "gxpo_tune": (ctypes.c_int, [_vp, ctypes.c_int, ctypes.c_int, ctypes.c_int]),
+    "gxpo_selftest_bounded_wait": (ctypes.c_int, [_vp, _vp]),
     "gxpo_launch_count": (ctypes.c_longlong, [_vp]),
     "gxpo_last_error": (ctypes.c_char_p, [_vp]),
     "gxpo_status_string": (ctypes.c_char_p, [ctypes.c_int]),
@@ -293,6 +294,10 @@ class Context:
 
     def tune(self, ctas_per_sm: int = 0, variant: int = 0, unit_tiles: int = 0):
         self._check(_lib.gxpo_tune(self._h, ctas_per_sm, variant, unit_tiles))
+
+    def selftest_bounded_wait(self, stream=None) -> int:
+        """Returns the status code (ERR_TIMEOUT is the expected outcome)."""
+        return _lib.gxpo_selftest_bounded_wait(self._h, _stream_ptr(stream))
 
     def launch_count(self) -> int:
         return _lib.gxpo_launch_count(self._h)

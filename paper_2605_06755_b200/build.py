@@ -10,7 +10,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libgxpo.so")
 SOURCES = [os.path.join(CSRC, "gxpo_api.cu")]
-DEPS = SOURCES + [os.path.join(CSRC, "gxpo_kernels.cuh"), os.path.join(ROOT, "include", "gxpo.h")]
+DEPS = SOURCES + [os.path.join(CSRC, "gxpo_kernels.cuh"), os.path.join(CSRC, "gxpo_bulk.cuh"), os.path.join(ROOT, "include", "gxpo.h")]
 
 
 def nvcc_path() -> str:

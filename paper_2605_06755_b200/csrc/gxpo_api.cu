@@ -2,6 +2,7 @@
 // machine of Algorithm 1, chunk tables and kernel launches.  C ABI in include/gxpo.h.
 #include "gxpo.h"
 #include "gxpo_kernels.cuh"
+#include "gxpo_bulk.cuh"
 
 #include <cmath>
 #include <cstdarg>
@@ -44,7 +45,9 @@ struct gxpo_ctx {
     int device;
     int sm_count;
     int ctas_per_sm;                   // 0 = default
-    int variant;                       // 1 = 128-bit, 2 = 256-bit
+    int variant;                       // 1 = 128-bit, 2 = 256-bit, 3 = 256-bit + bulk-copy staging of the fused sweep
+    int* d_err;                        // device error word (bounded waits)
+    int timeout_seen;
     int unit_shift;                    // work unit = kChunk >> unit_shift elements; -1 = choose per launch
     Phase phase;
     // bound list
@@ -208,6 +211,7 @@ typedef void (*FusedFn)(const TensorDesc*, const ChunkRef*, long long, TensorDes
                         double*, unsigned*, double*);
 
 StepFn pick_step(bool adamw, bool bf16, int variant) {
+    if (variant == 3) variant = 2;
     if (variant == 1) {
         if (adamw) return bf16 ? step_kernel<true, uint16_t, 4> : step_kernel<true, float, 4>;
         return bf16 ? step_kernel<false, uint16_t, 4> : step_kernel<false, float, 4>;
@@ -217,6 +221,7 @@ StepFn pick_step(bool adamw, bool bf16, int variant) {
 }
 // With diagnostics the sweeps use the 256-bit access variant only.
 ExtrapFn pick_extrap(bool bf16, int variant, bool diag) {
+    if (variant == 3) variant = 2;
     if (diag) return bf16 ? extrap_kernel<uint16_t, 8, true> : extrap_kernel<float, 8, true>;
     if (variant == 1) return bf16 ? extrap_kernel<uint16_t, 4, false> : extrap_kernel<float, 4, false>;
     return bf16 ? extrap_kernel<uint16_t, 8, false> : extrap_kernel<float, 8, false>;
@@ -270,6 +275,31 @@ gxpo_status launch_extrap(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, 
     return GXPO_OK;
 }
 
+// The bulk-copy staged variant of the fused sweep: one CTA per SM, whole chunks.
+typedef void (*BulkFn)(const TensorDesc*, const ChunkRef*, long long, TensorDesc, FusedParams, int*);
+template <bool ADAMW, typename G, bool DEFER>
+gxpo_status launch_bulk_t(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
+                          long long num_chunks, const TensorDesc& flat, const FusedParams& p) {
+    BulkFn fn = fused_bulk_kernel<ADAMW, G, DEFER>;
+    const int smem = (int)BulkLayout<ADAMW, G, DEFER>::kTotal;
+    CUDA_TRY(c, cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    long long g = c->sm_count;
+    if (g > num_chunks) g = num_chunks;
+    fn<<<(int)g, kBulkThreads, smem, s>>>(descs, chunks, num_chunks, flat, p, c->d_err);
+    c->launches += 1;
+    CUDA_TRY(c, cudaGetLastError());
+    return GXPO_OK;
+}
+gxpo_status launch_fused_bulk(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
+                              long long num_chunks, const TensorDesc& flat, const FusedParams& p, bool defer) {
+    const bool adamw = c->opt.kind == GXPO_OPT_ADAMW, bf16 = c->grad_dtype == GXPO_BF16;
+#define GXPO_BULK(A, G) (defer ? launch_bulk_t<A, G, true>(c, s, descs, chunks, num_chunks, flat, p) \
+                               : launch_bulk_t<A, G, false>(c, s, descs, chunks, num_chunks, flat, p))
+    if (adamw) return bf16 ? GXPO_BULK(true, uint16_t) : GXPO_BULK(true, float);
+    return bf16 ? GXPO_BULK(false, uint16_t) : GXPO_BULK(false, float);
+#undef GXPO_BULK
+}
+
 gxpo_status launch_fused(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
                          long long num_chunks, const TensorDesc& flat, const FusedParams& p, bool defer,
                          bool diag) {
@@ -277,7 +307,8 @@ gxpo_status launch_fused(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, c
         if (diag) CUDA_TRY(c, cudaMemsetAsync(c->d_diag, 0, (kDiagN + 1) * sizeof(double), s));
         return GXPO_OK;
     }
-    FusedFn fn = pick_fused(c->opt.kind == GXPO_OPT_ADAMW, c->grad_dtype == GXPO_BF16, c->variant, defer, diag);
+    if (c->variant == 3 && !diag) return launch_fused_bulk(c, s, descs, chunks, num_chunks, flat, p, defer);
+    FusedFn fn = pick_fused(c->opt.kind == GXPO_OPT_ADAMW, c->grad_dtype == GXPO_BF16, c->variant == 3 ? 2 : c->variant, defer, diag);
     const int ush = unit_shift_for(c, num_chunks);
     const int grid = grid_for(c, (const void*)fn, num_chunks << ush, kDefaultCtasFused);
     fn<<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, ush, c->d_diag_partials, c->d_ticket, c->d_diag);
@@ -310,7 +341,7 @@ void expire_clips(gxpo_ctx* c) {
 // t advances by one whatever the outcome, so the host mirror moves on at once.
 gxpo_status launch_gate(gxpo_ctx* c, cudaStream_t s, const double* sumsq) {
     gate_kernel<<<1, 32, 0, s>>>(c->d_gate, c->d_ring, sumsq, c->t, c->cfg.tau, c->cfg.gate_eps,
-                                 c->cfg.window, c->cfg.min_history, c->cfg.std_ddof, c->d_result);
+                                 c->cfg.window, c->cfg.min_history, c->cfg.std_ddof, c->d_err, c->d_result);
     c->launches += 1;
     CUDA_TRY(c, cudaGetLastError());
     CUDA_TRY(c, cudaMemcpyAsync(c->h_result, c->d_result, sizeof(GateResult), cudaMemcpyDeviceToHost, s));
@@ -327,6 +358,7 @@ gxpo_status finish_gate(gxpo_ctx* c) {
     c->gate_pending = 0;
     const GateResult r = *c->h_result;
     c->s_star = r.s_star;
+    if (r.dev_error) c->timeout_seen = 1;
     gxpo_gate_result& o = c->last_gate;
     o.active = r.active; o.tripped = r.tripped; o.t = r.t; o.s_star = r.s_star;
     o.norm = r.norm; o.z = r.z; o.mu = r.mu; o.sigma = r.sigma;
@@ -336,6 +368,10 @@ gxpo_status finish_gate(gxpo_ctx* c) {
 
 gxpo_status gate_outcome(gxpo_ctx* c, gxpo_gate_result* out) {
     if (out) *out = c->last_gate;
+    if (c->timeout_seen) {
+        c->timeout_seen = 0;
+        return fail(c, GXPO_ERR_TIMEOUT, "a bounded device-side wait gave up during step %lld: its outputs are incomplete", c->last_gate.t - 1);
+    }
     if (!std::isfinite(c->last_gate.norm))
         return fail(c, GXPO_ERR_NONFINITE, "||g_slow|| is not finite at step %lld; gate tripped", c->last_gate.t - 1);
     return GXPO_OK;
@@ -435,6 +471,8 @@ gxpo_status gxpo_create(const gxpo_cfg* cfg, const gxpo_opt_cfg* opt, int grad_d
     if (e == cudaSuccess) e = cudaMalloc(&c->d_partials, kMaxGrid * sizeof(double));
     if (e == cudaSuccess) e = cudaMalloc(&c->d_ticket, sizeof(unsigned));
     if (e == cudaSuccess) e = cudaMalloc(&c->d_sumsq, sizeof(double));
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_err, sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(c->d_err, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaMalloc(&c->d_gate, sizeof(GateState));
     if (e == cudaSuccess) e = cudaMalloc(&c->d_ring, (size_t)cfg->window * sizeof(double));
     if (e == cudaSuccess) e = cudaMalloc(&c->d_result, sizeof(GateResult));
@@ -471,6 +509,7 @@ void gxpo_destroy(gxpo_ctx* c) {
     cudaFree(c->d_partials);
     cudaFree(c->d_ticket);
     cudaFree(c->d_sumsq);
+    cudaFree(c->d_err);
     cudaFree(c->d_gate);
     cudaFree(c->d_ring);
     cudaFree(c->d_result);
@@ -788,6 +827,22 @@ gxpo_status gxpo_get_diagnostics(gxpo_ctx* c, void* stream, gxpo_diagnostics* ou
     return GXPO_OK;
 }
 
+gxpo_status gxpo_selftest_bounded_wait(gxpo_ctx* c, void* stream) {
+    if (!c) return GXPO_ERR_INVALID_ARG;
+    if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "self-test in the middle of a step");
+    cudaStream_t s = (cudaStream_t)stream;
+    bounded_wait_probe_kernel<<<1, 32, 0, s>>>(4096u, c->d_err);
+    c->launches += 1;
+    CUDA_TRY(c, cudaGetLastError());
+    int err = 0;
+    CUDA_TRY(c, cudaMemcpyAsync(&err, c->d_err, sizeof(int), cudaMemcpyDeviceToHost, s));
+    CUDA_TRY(c, cudaStreamSynchronize(s));
+    CUDA_TRY(c, cudaMemsetAsync(c->d_err, 0, sizeof(int), s));
+    CUDA_TRY(c, cudaStreamSynchronize(s));
+    if (err) return fail(c, GXPO_ERR_TIMEOUT, "self-test: the wait on a barrier nobody completes gave up, as it must");
+    return GXPO_OK;
+}
+
 gxpo_status gxpo_gate_peek(const gxpo_ctx* c, int* active, long long* s_star, long long* t) {
     if (!c) return GXPO_ERR_INVALID_ARG;
     { gxpo_status fg = finish_gate(const_cast<gxpo_ctx*>(c)); if (fg != GXPO_OK) return fg; }
@@ -826,7 +881,7 @@ const char* gxpo_status_string(gxpo_status s) {
 gxpo_status gxpo_tune(gxpo_ctx* c, int ctas_per_sm, int variant, int unit_tiles) {
     if (!c) return GXPO_ERR_INVALID_ARG;
     if (ctas_per_sm < 0 || ctas_per_sm > 16) return fail(c, GXPO_ERR_INVALID_ARG, "ctas_per_sm must be in [0, 16]");
-    if (variant < 0 || variant > 2) return fail(c, GXPO_ERR_INVALID_ARG, "variant must be 0, 1 or 2");
+    if (variant < 0 || variant > 3) return fail(c, GXPO_ERR_INVALID_ARG, "variant must be 0, 1, 2 or 3");
     int ush = -1;
     const bool auto_unit = unit_tiles == 0;
     if (auto_unit) ush = 0;

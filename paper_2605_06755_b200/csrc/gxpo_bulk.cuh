@@ -1,0 +1,250 @@
+// Bulk-copy (TMA) staging for the fused probe + extrapolate sweep: an alternative to the
+// register-staged kernel, kept selectable (gxpo_tune variant 3) because it is the design
+// one would expect to win on this GPU and the measurement says otherwise.
+//
+// One producer thread streams whole 2048-element tiles of every input array into a
+// shared-memory ring with cp.async.bulk (no tensor map, no multicast, this GPU's own
+// memory only); eight consumer warps pick a tile up when its mbarrier completes, do the
+// same per-coordinate arithmetic as the register-staged kernel (same functions, hence the
+// same bits) and store straight from registers.  Up to kStages - 1 tiles per SM are in
+// flight whatever the consumers are doing.
+//
+// Every wait on an mbarrier is bounded: after kWaitLimit polls the waiting thread raises
+// the kernel's error word, tells the rest of the CTA to stop, and returns; the host then
+// reports GXPO_ERR_TIMEOUT.  A producer that gives up first waits (bounded again) for the
+// copies it already issued, so that none lands in shared memory after the CTA has gone.
+#pragma once
+
+#include "gxpo_kernels.cuh"
+
+namespace gxpo {
+
+constexpr int kStages = 4;
+constexpr int kConsumerWarps = kThreads / 32;
+constexpr int kBulkThreads = kThreads + 32;         // consumers + one producer warp
+constexpr unsigned kWaitLimit = 1u << 22;           // polls per wait (each poll may itself block briefly)
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity) {
+    unsigned ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// false = gave up after `limit` polls, or another thread of the CTA already did
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, unsigned parity, volatile int* stop,
+                                                  unsigned limit) {
+    for (unsigned i = 0; i < limit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*stop) return false;
+        if (i > 1024) __nanosleep(64);
+    }
+    return false;
+}
+// global -> this CTA's shared memory; src, dst and size are multiples of 16 bytes
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, unsigned bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ FVec<8> lds_f8(const float* p) {
+    FVec<8> r;
+    const uint32_t a = smem_u32(p);
+    // "memory": these reads must stay ahead of the arrive that hands the stage back
+    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(r.x[0]), "=f"(r.x[1]), "=f"(r.x[2]), "=f"(r.x[3]) : "r"(a) : "memory");
+    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(r.x[4]), "=f"(r.x[5]), "=f"(r.x[6]), "=f"(r.x[7]) : "r"(a + 16) : "memory");
+    return r;
+}
+__device__ __forceinline__ FVec<8> lds_g8(const float* p) { return lds_f8(p); }
+__device__ __forceinline__ FVec<8> lds_g8(const uint16_t* p) {
+    HVec<8> h;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(h.x[0]), "=r"(h.x[1]), "=r"(h.x[2]), "=r"(h.x[3]) : "r"(smem_u32(p)) : "memory");
+    FVec<8> r;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { r.x[2 * i] = bf16_lo(h.x[i]); r.x[2 * i + 1] = bf16_hi(h.x[i]); }
+    return r;
+}
+
+// one chunk of one tensor, pointers resolved
+template <typename G> struct FusedUnit {
+    const float* t1; const float* t0; float* out; float* m; float* v; const G* g0; const G* g1;
+    uint16_t* wb;
+    int len, full_tiles;                // full_tiles > 0 only when every pointer is 32-byte aligned
+    bool vec;
+};
+
+template <bool ADAMW, typename G, bool DEFER>
+__device__ __forceinline__ bool fused_resolve(long long c, const TensorDesc* descs, const ChunkRef* chunks,
+                                              const TensorDesc& flat, const FusedParams& p, FusedUnit<G>& U) {
+    ChunkRef ref;
+    TensorDesc d;
+    if (chunks) { ref = chunks[c]; d = descs[ref.tensor]; }
+    else { ref.tensor = 0; ref.chunk = (unsigned)c; d = flat; }
+    const long long off = (long long)ref.chunk * kChunk;
+    const long long rem = d.n - off;
+    U.len = 0; U.full_tiles = 0; U.vec = false;
+    if (rem <= 0) return false;
+    U.len = rem < kChunk ? (int)rem : kChunk;
+    U.t1 = (p.step.in_sel ? d.work : d.theta) + off;
+    U.t0 = (p.ex.theta0_sel ? d.work : d.theta) + off;
+    U.out = d.theta + off;
+    U.m = ADAMW ? d.m + off : nullptr;
+    U.v = ADAMW ? d.v + off : nullptr;
+    U.g0 = reinterpret_cast<const G*>(d.g[0]) + off;
+    U.g1 = reinterpret_cast<const G*>(d.g[1]) + off;
+    U.wb = d.wb ? d.wb + off : nullptr;
+    U.vec = (DEFER || aligned32(U.t1)) && aligned32(U.t0) && aligned32(U.out) && aligned32(U.g0) &&
+            aligned32(U.g1) && (!ADAMW || (aligned32(U.m) && aligned32(U.v))) && aligned16(U.wb);
+    U.full_tiles = U.vec ? U.len / kTile : 0;
+    return true;
+}
+
+// Shared memory per stage: [theta1 unless DEFER] theta0 [m v if ADAMW] g0 g1, one tile each.
+template <bool ADAMW, typename G, bool DEFER>
+struct BulkLayout {
+    static constexpr unsigned kF = kTile * sizeof(float);
+    static constexpr unsigned kGb = kTile * sizeof(G);
+    static constexpr unsigned kStage = ((DEFER ? 1 : 2) + (ADAMW ? 2 : 0)) * kF + 2 * kGb;
+    static constexpr unsigned kTotal = kStages * kStage + 2 * kStages * sizeof(uint64_t) + 16;
+};
+
+template <bool ADAMW, typename G, bool DEFER>
+__global__ void __launch_bounds__(kBulkThreads, 1)
+fused_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restrict__ chunks,
+                  long long num_chunks, TensorDesc flat, FusedParams p, int* error_word) {
+    typedef BulkLayout<ADAMW, G, DEFER> L;
+    extern __shared__ __align__(128) unsigned char smem[];
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStages * L::kStage);
+    uint64_t* empty = full + kStages;
+    volatile int* stop = reinterpret_cast<volatile int*>(empty + kStages);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, kConsumerWarps); }
+        *stop = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (warp == kConsumerWarps) {                       // ---- producer warp: lane 0 issues the copies
+        if (lane != 0) return;
+        unsigned it = 0;
+        bool ok = true;
+        for (long long c = blockIdx.x; c < num_chunks && ok; c += gridDim.x) {
+            FusedUnit<G> U;
+            if (!fused_resolve<ADAMW, G, DEFER>(c, descs, chunks, flat, p, U)) continue;
+            for (int j = 0; j < U.full_tiles; ++j, ++it) {
+                const unsigned s = it % kStages, n = it / kStages;
+                // the consumers must have released the stage's previous use
+                if (n > 0 && !mbar_wait_bounded(empty + s, (n - 1) & 1, stop, kWaitLimit)) { ok = false; break; }
+                unsigned char* st = smem + s * L::kStage;
+                const int e = j * kTile;
+                mbar_expect_tx(full + s, L::kStage);
+                unsigned o = 0;
+                if (!DEFER) { bulk_load(st, U.t1 + e, L::kF, full + s); o += L::kF; }
+                bulk_load(st + o, U.t0 + e, L::kF, full + s); o += L::kF;
+                if (ADAMW) {
+                    bulk_load(st + o, U.m + e, L::kF, full + s); o += L::kF;
+                    bulk_load(st + o, U.v + e, L::kF, full + s); o += L::kF;
+                }
+                bulk_load(st + o, U.g0 + e, L::kGb, full + s); o += L::kGb;
+                bulk_load(st + o, U.g1 + e, L::kGb, full + s);
+            }
+        }
+        if (!ok) {
+            *stop = 1;
+            atomicExch(error_word, 1);
+            // copies already issued still target this CTA's shared memory: give each of the
+            // last kStages uses a bounded chance to land before the CTA goes away
+            for (unsigned k = 0; k < (unsigned)kStages && k < it; ++k) {
+                const unsigned i2 = it - 1 - k;
+                for (unsigned w = 0; w < kWaitLimit && !mbar_try_wait(full + i2 % kStages, (i2 / kStages) & 1); ++w)
+                    __nanosleep(64);
+            }
+        }
+        return;
+    }
+
+    // ---- consumers
+    const float gs0 = p.ex.gscale0 ? __ldg(p.ex.gscale0) : 1.0f, gs1 = p.ex.gscale1 ? __ldg(p.ex.gscale1) : 1.0f;
+    unsigned it = 0;
+    for (long long c = blockIdx.x; c < num_chunks; c += gridDim.x) {
+        FusedUnit<G> U;
+        if (!fused_resolve<ADAMW, G, DEFER>(c, descs, chunks, flat, p, U)) continue;
+        if (!U.vec) {                                   // misaligned tensor: scalar path, no staging
+            for (int e = threadIdx.x; e < U.len; e += kThreads) {
+                float mm = ADAMW ? U.m[e] : 0.0f, vv = ADAMW ? U.v[e] : 0.0f;
+                const float x = fused_elem<ADAMW, DEFER, false>(DEFER ? 0.0f : U.t1[e], U.t0[e], mm, vv,
+                                                                __fmul_rn(ld_grad1(U.g0 + e), gs0),
+                                                                __fmul_rn(ld_grad1(U.g1 + e), gs1), p, nullptr);
+                U.out[e] = x;
+                if (U.wb) U.wb[e] = to_bf16(x);
+                if (ADAMW) { U.m[e] = mm; U.v[e] = vv; }
+            }
+            continue;
+        }
+        for (int j = 0; j < U.full_tiles; ++j, ++it) {
+            const unsigned s = it % kStages, n = it / kStages;
+            if (!mbar_wait_bounded(full + s, n & 1, stop, kWaitLimit)) {
+                *stop = 1;
+                atomicExch(error_word, 1);
+                return;
+            }
+            const unsigned char* st = smem + s * L::kStage;
+            const int tt = threadIdx.x * 8;
+            unsigned o = 0;
+            FVec<8> a1, a0, mm, vv;
+            if (!DEFER) { a1 = lds_f8(reinterpret_cast<const float*>(st) + tt); o += L::kF; }
+            a0 = lds_f8(reinterpret_cast<const float*>(st + o) + tt); o += L::kF;
+            if (ADAMW) {
+                mm = lds_f8(reinterpret_cast<const float*>(st + o) + tt); o += L::kF;
+                vv = lds_f8(reinterpret_cast<const float*>(st + o) + tt); o += L::kF;
+            }
+            FVec<8> b0 = scaled<8>(lds_g8(reinterpret_cast<const G*>(st + o) + tt), gs0); o += L::kGb;
+            FVec<8> b1 = scaled<8>(lds_g8(reinterpret_cast<const G*>(st + o) + tt), gs1);
+            const int e = j * kTile + tt;
+            if (DEFER) {
+                a1 = a0;
+                optim_step_vec<ADAMW, 8>(a1, mm, vv, b0, p.step0);
+            }
+            optim_step_vec<ADAMW, 8>(a1, mm, vv, b1, p.step);
+            extrapolate_vec<8, false>(a1, a0, b0, b1, p.ex, nullptr);
+            st_f(U.out + e, a1);
+            if (U.wb) st_bf16(U.wb + e, a1);
+            if (ADAMW) { st_f(U.m + e, mm); st_f(U.v + e, vv); }
+            // Hand the stage back only now: every lane's stores depend on what it read from
+            // the stage, so by this point the shared-memory reads have certainly completed.
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty + s);
+        }
+        // ragged rest of the chunk (less than one tile): register path
+        const int done = U.full_tiles * kTile;
+        if (done < U.len)
+            fused_chunk_vec<ADAMW, G, 8, DEFER, false>(U.out + done, U.t1 + done, U.t0 + done,
+                                                       ADAMW ? U.m + done : nullptr, ADAMW ? U.v + done : nullptr,
+                                                       U.g0 + done, U.g1 + done, U.len - done, p, gs0, gs1, nullptr,
+                                                       U.wb ? U.wb + done : nullptr);
+    }
+}
+
+// Nothing ever completes the barrier this kernel waits on: the bounded wait has to give up
+// after `limit` polls and raise the error word.  Used to check that path end to end.
+__global__ void bounded_wait_probe_kernel(unsigned limit, int* error_word) {
+    __shared__ uint64_t bar;
+    __shared__ int stop_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        stop_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (!mbar_wait_bounded(&bar, 0, &stop_flag, limit)) atomicExch(error_word, 1);
+    }
+}
+
+}  // namespace gxpo

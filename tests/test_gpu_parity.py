@@ -232,7 +232,7 @@ def test_access_variants_and_launch_shapes_agree_bitwise():
     b = _binding()
     n = 5 * 32768 + 77
     outs = []
-    for variant, ctas, unit in [(1, 0, 0), (2, 0, 0), (2, 1, 1), (1, 7, 4), (2, 3, 16), (2, 2, 2)]:
+    for variant, ctas, unit in [(1, 0, 0), (2, 0, 0), (2, 1, 1), (1, 7, 4), (2, 3, 16), (2, 2, 2), (3, 0, 0)]:
         pr = _problem(n, seed=42, grad_dtype="bf16")
         ctx, cfg, opt = _ctx(b, "bf16", lr=1e-3, K=5)
         ctx.tune(ctas, variant, unit)
@@ -453,4 +453,53 @@ def test_no_sweep_writes_outside_its_tensors(flow, placement):
         assert torch.equal(pr.g0.view(torch.int16), g0.view(torch.int16))
         assert torch.equal(pr.g1.view(torch.int16), g1.view(torch.int16))
         assert torch.equal(pr.gs.view(torch.int16), gs.view(torch.int16))
+    ctx.close()
+
+
+@pytest.mark.parametrize("kind,grad_dtype", [("adamw", "bf16"), ("adamw", "f32"), ("gd", "f32"), ("gd", "bf16")])
+@pytest.mark.parametrize("deferred", [False, True])
+def test_bulk_copy_staged_fused_sweep_is_bit_identical(kind, grad_dtype, deferred):
+    """Variant 3 (tiles staged in shared memory by bulk asynchronous copies) against the
+    register-staged sweep: full tiles, ragged chunk ends, a misaligned tensor, tensors
+    smaller than a tile, many chunks per CTA, gradient scales and bfloat16 copies on."""
+    import torch
+    b = _binding()
+    sizes = [40 * 32768 + 5, 2047, 1, 40003, 2048, 3 * 2048 + 17, 300 * 32768]
+    offsets = [0, 0, 0, 1, 0, 0, 0]
+    outs = []
+    for variant in (2, 3):
+        probs = [_problem(n, seed=90 + i, grad_dtype=grad_dtype, zero_frac=0.03, offset=off)
+                 for i, (n, off) in enumerate(zip(sizes, offsets))]
+        ctx, cfg, opt = _ctx(b, grad_dtype, kind=b.OPT_ADAMW if kind == "adamw" else b.OPT_GD, lr=1e-3, K=5, alpha=0.5)
+        ctx.tune(0, variant, 0)
+        ctx.bind([p.ptrs() for p in probs])
+        wbs = [torch.zeros(p.n, dtype=torch.bfloat16, device="cuda") for p in probs]
+        ctx.bind_model_weights([w.data_ptr() for w in wbs])
+        scales = torch.tensor([0.5, 0.75, 1.0], dtype=torch.float32, device="cuda")
+        for k in range(3):
+            ctx.set_grad_scale(k, scales.data_ptr() + 4 * k)
+        rec = []
+        for _ in range(2):
+            res = ctx.active_step(allow_nonfinite=True, fused=not deferred, deferred=deferred)
+            rec += [gu.to_host_f64(p.theta) for p in probs] + [gu.to_host_f64(p.m) for p in probs]
+            rec += [gu.to_host_f64(p.v) for p in probs] + [gu.to_host_f64(w) for w in wbs] + [np.array(res.norm)]
+        outs.append(rec)
+        ctx.close()
+    for x, y in zip(outs[0], outs[1]):
+        np.testing.assert_array_equal(x, y)
+
+
+def test_bounded_wait_gives_up_and_reports_timeout():
+    """A wait on a barrier that nothing completes must end by itself, raise the device
+    error word and leave the context usable."""
+    b = _binding()
+    pr = _problem(5000, 3, "bf16")
+    ctx, cfg, opt = _ctx(b, "bf16", lr=1e-3)
+    ctx.bind([pr.ptrs()])
+    assert ctx.selftest_bounded_wait() == b.ERR_TIMEOUT
+    assert "gave up" in b._lib.gxpo_last_error(ctx._h).decode()
+    res = ctx.active_step(allow_nonfinite=True, deferred=True)     # still works, and the word was cleared
+    assert res.t == 1
+    ctx.tune(0, 3, 0)
+    assert ctx.active_step(allow_nonfinite=True, deferred=True).t == 2
     ctx.close()
