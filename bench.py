@@ -101,19 +101,24 @@ def measured_peak_gbs():
 
 def recorded_traffic_per_param(kernel_fn, calls):
     """DRAM bytes per parameter of `kernel_fn`, averaged over the named calls, from the
-    committed ncu summary profiles/<kernel_fn>_adamw_bf16_flat134m.txt (lines
+    committed ncu summary profiles/<kernel_fn>_adamw_bf16_flat*.txt (lines
     "dram_bytes_per_param[<call>]: X").  The summary records the hash of the kernel source
     it was taken from; once that source has changed the counters no longer describe the
     kernel and None is returned."""
     import hashlib
     import re
-    summary = os.path.join(ROOT, "profiles", f"{kernel_fn}_adamw_bf16_flat134m.txt")
+    import glob
     source = os.path.join(ROOT, "paper_2605_06755_b200", "csrc", "gxpo_kernels.cuh")
     try:
+        summary = sorted(glob.glob(os.path.join(ROOT, "profiles", f"{kernel_fn}_adamw_bf16_flat*.txt")))[0]
         text = open(summary).read()
         want = re.search(r"^kernel_source_sha256:\s*([0-9a-f]{64})", text, re.M).group(1)
         have = hashlib.sha256(open(source, "rb").read()).hexdigest()
         if have != want:
+            return None
+        bulk = re.search(r"^bulk_source_sha256:\s*([0-9a-f]{64})", text, re.M)
+        if bulk and bulk.group(1) != hashlib.sha256(
+                open(os.path.join(os.path.dirname(source), "gxpo_bulk.cuh"), "rb").read()).hexdigest():
             return None
         vals = [float(re.search(r"^dram_bytes_per_param\[%s\]:\s*([0-9.]+)" % re.escape(c), text, re.M).group(1))
                 for c in calls]
@@ -393,13 +398,18 @@ def run_ours(args):
         alg_bytes["probe_step0_deferred"] -= 2
         alg_bytes["probe_extrapolate_deferred"] += 2
         alg_bytes["slow_step"] += 2
-    kernels = {nm: {"kernel": KERNEL_OF[nm], "ms": ms, "bytes_per_param": alg_bytes[nm],
+    kernel_of = dict(KERNEL_OF)
+    n_chunks = sum((k + 32767) // 32768 for _, k in shapes)
+    if args.variant == 3 or (args.variant == 0 and n_chunks >= 32 * props.multi_processor_count):
+        # the fused sweep runs in its bulk-copy staged kernel (the library's default for long lists)
+        kernel_of["probe_extrapolate"] = kernel_of["probe_extrapolate_deferred"] = "fused_bulk_kernel"
+    kernels = {nm: {"kernel": kernel_of[nm], "ms": ms, "bytes_per_param": alg_bytes[nm],
                     "gbs": alg_bytes[nm] * d / (ms * 1e-3) / 1e9} for nm, ms in per.items()}
     # dominant kernel = the kernel function with the largest share of the step; its figures
     # are averages over its launches in one step (algorithmic bytes and duration alike)
     by_fn = {}
     for nm, ms in per.items():
-        by_fn.setdefault(KERNEL_OF[nm], []).append(nm)
+        by_fn.setdefault(kernel_of[nm], []).append(nm)
     dom_fn = max(by_fn, key=lambda f: sum(per[nm] for nm in by_fn[f]))
     dom = by_fn[dom_fn]
     dom_bytes = statistics.mean(alg_bytes[nm] for nm in dom) * d

@@ -20,6 +20,7 @@ constexpr int kDefaultCtasStep = 2;    // measured best for the 14R/12W sweep
 constexpr int kDefaultCtasStepLight = 3;  // 14R/4W (deferred first probe): read-heavy, wants more loads in flight
 constexpr int kDefaultCtasExtrap = 4;  // the extrapolation needs more warps to cover its arithmetic
 constexpr int kDefaultCtasFused = 3;
+constexpr int kDefaultCtasBulk = 1;    // one CTA per SM with a 3-stage ring measured best (2 is as good, 4+ stages worse)
 
 enum Phase { IDLE = 0, PROBED0 = 1, PROBED1 = 2, EXTRAPOLATED = 3, SLOW_DONE = 4, PROBED0_DEFERRED = 5 };
 
@@ -45,7 +46,7 @@ struct gxpo_ctx {
     int device;
     int sm_count;
     int ctas_per_sm;                   // 0 = default
-    int variant;                       // 1 = 128-bit, 2 = 256-bit, 3 = 256-bit + bulk-copy staging of the fused sweep
+    int variant;                       // 0 = default, 1 = 128-bit, 2 = 256-bit register staging, 3 = 256-bit + bulk-copy staged fused sweep
     int* d_err;                        // device error word (bounded waits)
     int timeout_seen;
     int unit_shift;                    // work unit = kChunk >> unit_shift elements; -1 = choose per launch
@@ -211,7 +212,7 @@ typedef void (*FusedFn)(const TensorDesc*, const ChunkRef*, long long, TensorDes
                         double*, unsigned*, double*);
 
 StepFn pick_step(bool adamw, bool bf16, int variant) {
-    if (variant == 3) variant = 2;
+    if (variant != 1) variant = 2;
     if (variant == 1) {
         if (adamw) return bf16 ? step_kernel<true, uint16_t, 4> : step_kernel<true, float, 4>;
         return bf16 ? step_kernel<false, uint16_t, 4> : step_kernel<false, float, 4>;
@@ -221,7 +222,7 @@ StepFn pick_step(bool adamw, bool bf16, int variant) {
 }
 // With diagnostics the sweeps use the 256-bit access variant only.
 ExtrapFn pick_extrap(bool bf16, int variant, bool diag) {
-    if (variant == 3) variant = 2;
+    if (variant != 1) variant = 2;
     if (diag) return bf16 ? extrap_kernel<uint16_t, 8, true> : extrap_kernel<float, 8, true>;
     if (variant == 1) return bf16 ? extrap_kernel<uint16_t, 4, false> : extrap_kernel<float, 4, false>;
     return bf16 ? extrap_kernel<uint16_t, 8, false> : extrap_kernel<float, 8, false>;
@@ -283,7 +284,12 @@ gxpo_status launch_bulk_t(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, 
     BulkFn fn = fused_bulk_kernel<ADAMW, G, DEFER>;
     const int smem = (int)BulkLayout<ADAMW, G, DEFER>::kTotal;
     CUDA_TRY(c, cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    long long g = c->sm_count;
+    int resident = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, (const void*)fn, kBulkThreads, (size_t)smem) != cudaSuccess || resident < 1)
+        resident = 1;
+    int per_sm = c->ctas_per_sm > 0 ? c->ctas_per_sm : kDefaultCtasBulk;
+    if (per_sm > resident) per_sm = resident;
+    long long g = (long long)c->sm_count * per_sm;
     if (g > num_chunks) g = num_chunks;
     fn<<<(int)g, kBulkThreads, smem, s>>>(descs, chunks, num_chunks, flat, p, c->d_err);
     c->launches += 1;
@@ -307,8 +313,14 @@ gxpo_status launch_fused(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, c
         if (diag) CUDA_TRY(c, cudaMemsetAsync(c->d_diag, 0, (kDiagN + 1) * sizeof(double), s));
         return GXPO_OK;
     }
-    if (c->variant == 3 && !diag) return launch_fused_bulk(c, s, descs, chunks, num_chunks, flat, p, defer);
-    FusedFn fn = pick_fused(c->opt.kind == GXPO_OPT_ADAMW, c->grad_dtype == GXPO_BF16, c->variant == 3 ? 2 : c->variant, defer, diag);
+    // default (0): the bulk-copy staged kernel for lists long enough to keep every SM's ring
+    // busy (it deals whole chunks, one CTA per SM), register staging for short lists; 3
+    // forces bulk staging, 1 and 2 force register staging.  Diagnostics exist only in the
+    // register-staged kernel.
+    const bool long_list = num_chunks >= 32LL * c->sm_count;
+    if (((c->variant == 0 && long_list) || c->variant == 3) && !diag)
+        return launch_fused_bulk(c, s, descs, chunks, num_chunks, flat, p, defer);
+    FusedFn fn = pick_fused(c->opt.kind == GXPO_OPT_ADAMW, c->grad_dtype == GXPO_BF16, c->variant == 1 ? 1 : 2, defer, diag);
     const int ush = unit_shift_for(c, num_chunks);
     const int grid = grid_for(c, (const void*)fn, num_chunks << ush, kDefaultCtasFused);
     fn<<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, ush, c->d_diag_partials, c->d_ticket, c->d_diag);
@@ -462,7 +474,7 @@ gxpo_status gxpo_create(const gxpo_cfg* cfg, const gxpo_opt_cfg* opt, int grad_d
     c->cfg = *cfg;
     c->opt = *opt;
     c->grad_dtype = grad_dtype;
-    c->variant = 2;
+    c->variant = 0;
     c->unit_shift = -1;
     c->s_star = -1;
     c->phase = IDLE;
@@ -888,7 +900,7 @@ gxpo_status gxpo_tune(gxpo_ctx* c, int ctas_per_sm, int variant, int unit_tiles)
     for (int k = 0; k <= 4; ++k) if (unit_tiles == (kTilesPerChunk >> k)) ush = k;
     if (ush < 0) return fail(c, GXPO_ERR_INVALID_ARG, "unit_tiles must be 0, 1, 2, 4, 8 or 16");
     c->ctas_per_sm = ctas_per_sm;
-    c->variant = variant == 0 ? 2 : variant;
+    c->variant = variant;
     c->unit_shift = auto_unit ? -1 : ush;
     return GXPO_OK;
 }

@@ -19,7 +19,10 @@
 
 namespace gxpo {
 
-constexpr int kStages = 4;
+#ifndef GXPO_BULK_STAGES
+#define GXPO_BULK_STAGES 3
+#endif
+constexpr int kStages = GXPO_BULK_STAGES;
 constexpr int kConsumerWarps = kThreads / 32;
 constexpr int kBulkThreads = kThreads + 32;         // consumers + one producer warp
 constexpr unsigned kWaitLimit = 1u << 22;           // polls per wait (each poll may itself block briefly)
