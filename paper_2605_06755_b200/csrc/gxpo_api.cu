@@ -283,10 +283,17 @@ gxpo_status launch_bulk_t(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, 
                           long long num_chunks, const TensorDesc& flat, const FusedParams& p) {
     BulkFn fn = fused_bulk_kernel<ADAMW, G, DEFER>;
     const int smem = (int)BulkLayout<ADAMW, G, DEFER>::kTotal;
-    CUDA_TRY(c, cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    int resident = 1;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, (const void*)fn, kBulkThreads, (size_t)smem) != cudaSuccess || resident < 1)
-        resident = 1;
+    // first launch of this instantiation in this context: allow the ring's shared memory and
+    // find out how many CTAs fit; remembered in the occupancy cache afterwards
+    int resident = 0;
+    for (int i = 0; i < c->occ_n; ++i)
+        if (c->occ_key[i] == (const void*)fn) resident = c->occ_val[i];
+    if (resident == 0) {
+        CUDA_TRY(c, cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, (const void*)fn, kBulkThreads, (size_t)smem) != cudaSuccess || resident < 1)
+            resident = 1;
+        if (c->occ_n < 32) { c->occ_key[c->occ_n] = (const void*)fn; c->occ_val[c->occ_n] = resident; c->occ_n += 1; }
+    }
     int per_sm = c->ctas_per_sm > 0 ? c->ctas_per_sm : kDefaultCtasBulk;
     if (per_sm > resident) per_sm = resident;
     long long g = (long long)c->sm_count * per_sm;
