@@ -303,3 +303,51 @@ def test_async_gate_update_gives_the_same_decisions():
         asyn.probe_step_deferred()                       # tripped: the active phase is over
     assert e.value.status == b.ERR_STATE
     sync.close(); asyn.close()
+
+
+def test_two_contexts_on_two_streams_and_rebinding():
+    """Contexts own their scratch, so two of them may run at the same time on different
+    streams; and a context may be re-bound to another list between steps.  Results must be
+    those of the same steps run one after the other."""
+    import torch
+    b = _binding()
+    sizes = [5 * 32768 + 77, 70001]
+
+    def fresh(seed):
+        probs = _small_list(b, sizes, seed=seed)
+        cfg, opt = b.make_cfg(lr=1e-3, K=5, alpha=0.5)
+        ctx = b.Context(cfg, opt, b.BF16)
+        ctx.bind([p.ptrs() for p in probs])
+        return probs, ctx
+
+    # serial reference
+    ref = []
+    for seed in (11, 12):
+        probs, ctx = fresh(seed)
+        for _ in range(3):
+            r = ctx.active_step(deferred=True)
+        ref.append(([gu.to_host_f64(p.theta) for p in probs], r.norm))
+        ctx.close()
+    # the same two runs interleaved on two streams
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    (p1, c1), (p2, c2) = fresh(11), fresh(12)
+    torch.cuda.synchronize()
+    for _ in range(3):
+        c1.probe_step_deferred(s1); c2.probe_step_deferred(s2)
+        c1.probe_extrapolate(s1); c2.probe_extrapolate(s2)
+        c1.slow_step(s1); c2.slow_step(s2)
+        c1.gate_update_async(s1); c2.gate_update_async(s2)
+    r1, r2 = c1.gate_last(), c2.gate_last()
+    torch.cuda.synchronize()
+    for probs, r, (want, norm) in ((p1, r1, ref[0]), (p2, r2, ref[1])):
+        for p, w in zip(probs, want):
+            np.testing.assert_array_equal(gu.to_host_f64(p.theta), w)
+        assert r.norm == norm
+    # re-bind c1 to the second list's tensors (state carries over, data is the caller's)
+    c1.bind([p.ptrs() for p in p2])
+    before = [gu.to_host_f64(p.theta) for p in p2]
+    c1.active_step(deferred=True)
+    assert c1.optimizer_steps() == 12 and c1.gate_peek()[2] == 4
+    assert any(not np.array_equal(gu.to_host_f64(p.theta), x) for p, x in zip(p2, before))
+    c1.close(); c2.close()
