@@ -2,12 +2,12 @@
 // register-staged kernel, kept selectable (gxpo_tune variant 3) because it is the design
 // one would expect to win on this GPU and the measurement says otherwise.
 //
-// One producer thread streams whole 2048-element tiles of every input array into a
-// shared-memory ring with cp.async.bulk (no tensor map, no multicast, this GPU's own
+// One producer thread streams whole stages (one or two 2048-element tiles of every input
+// array) into a shared-memory ring with cp.async.bulk (no tensor map, no multicast, this GPU's own
 // memory only); eight consumer warps pick a tile up when its mbarrier completes, do the
 // same per-coordinate arithmetic as the register-staged kernel (same functions, hence the
-// same bits) and store straight from registers.  Up to kStages - 1 tiles per SM are in
-// flight whatever the consumers are doing.
+// same bits) and store straight from registers.  All but one stage of the ring are in flight
+// whatever the consumers are doing.
 //
 // Every wait on an mbarrier is bounded: after kWaitLimit polls the waiting thread raises
 // the kernel's error word, tells the rest of the CTA to stop, and returns; the host then
@@ -19,10 +19,7 @@
 
 namespace gxpo {
 
-#ifndef GXPO_BULK_STAGES
-#define GXPO_BULK_STAGES 3
-#endif
-constexpr int kStages = GXPO_BULK_STAGES;
+constexpr int kMaxStages = 3;
 constexpr int kConsumerWarps = kThreads / 32;
 constexpr int kBulkThreads = kThreads + 32;         // consumers + one producer warp
 constexpr unsigned kWaitLimit = 1u << 22;           // polls per wait (each poll may itself block briefly)
@@ -86,7 +83,8 @@ template <typename G> struct FusedUnit {
 
 template <bool ADAMW, typename G, bool DEFER>
 __device__ __forceinline__ bool fused_resolve(long long c, const TensorDesc* descs, const ChunkRef* chunks,
-                                              const TensorDesc& flat, const FusedParams& p, FusedUnit<G>& U) {
+                                              const TensorDesc& flat, const FusedParams& p, int stage_elems,
+                                              FusedUnit<G>& U) {
     ChunkRef ref;
     TensorDesc d;
     if (chunks) { ref = chunks[c]; d = descs[ref.tensor]; }
@@ -106,17 +104,24 @@ __device__ __forceinline__ bool fused_resolve(long long c, const TensorDesc* des
     U.wb = d.wb ? d.wb + off : nullptr;
     U.vec = (DEFER || aligned32(U.t1)) && aligned32(U.t0) && aligned32(U.out) && aligned32(U.g0) &&
             aligned32(U.g1) && (!ADAMW || (aligned32(U.m) && aligned32(U.v))) && aligned16(U.wb);
-    U.full_tiles = U.vec ? U.len / kTile : 0;
+    U.full_tiles = U.vec ? U.len / stage_elems : 0;
     return true;
 }
 
-// Shared memory per stage: [theta1 unless DEFER] theta0 [m v if ADAMW] g0 g1, one tile each.
+// Shared memory per stage: [theta1 unless DEFER] theta0 [m v if ADAMW] g0 g1, kMult tiles each.
+// Ring shape, measured on a 7.6e9-parameter list: what matters is about 64 KB in flight per SM
+// in as few, as large pieces as possible.  Deferred sweep (5 arrays): 2 stages of 4096
+// elements 6.62 TB/s, 3 of 2048 6.53, 2 of 2048 5.77, 4 of 2048 6.10, 3 of 4096 6.09.  The
+// non-deferred sweep (6 arrays) does best with 3 stages of 2048.
 template <bool ADAMW, typename G, bool DEFER>
 struct BulkLayout {
-    static constexpr unsigned kF = kTile * sizeof(float);
-    static constexpr unsigned kGb = kTile * sizeof(G);
+    static constexpr int kMult = DEFER ? 2 : 1;                  // tiles per stage
+    static constexpr int kStagesN = DEFER ? 2 : 3;
+    static constexpr int kElems = kTile * kMult;
+    static constexpr unsigned kF = kElems * sizeof(float);
+    static constexpr unsigned kGb = kElems * sizeof(G);
     static constexpr unsigned kStage = ((DEFER ? 1 : 2) + (ADAMW ? 2 : 0)) * kF + 2 * kGb;
-    static constexpr unsigned kTotal = kStages * kStage + 2 * kStages * sizeof(uint64_t) + 16;
+    static constexpr unsigned kTotal = kStagesN * kStage + 2 * kMaxStages * sizeof(uint64_t) + 16;
 };
 
 template <bool ADAMW, typename G, bool DEFER>
@@ -125,9 +130,10 @@ fused_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restri
                   long long num_chunks, TensorDesc flat, FusedParams p, int* error_word) {
     typedef BulkLayout<ADAMW, G, DEFER> L;
     extern __shared__ __align__(128) unsigned char smem[];
+    constexpr int kStages = L::kStagesN;
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStages * L::kStage);
-    uint64_t* empty = full + kStages;
-    volatile int* stop = reinterpret_cast<volatile int*>(empty + kStages);
+    uint64_t* empty = full + kMaxStages;
+    volatile int* stop = reinterpret_cast<volatile int*>(empty + kMaxStages);
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, kConsumerWarps); }
         *stop = 0;
@@ -142,13 +148,13 @@ fused_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restri
         bool ok = true;
         for (long long c = blockIdx.x; c < num_chunks && ok; c += gridDim.x) {
             FusedUnit<G> U;
-            if (!fused_resolve<ADAMW, G, DEFER>(c, descs, chunks, flat, p, U)) continue;
+            if (!fused_resolve<ADAMW, G, DEFER>(c, descs, chunks, flat, p, L::kElems, U)) continue;
             for (int j = 0; j < U.full_tiles; ++j, ++it) {
                 const unsigned s = it % kStages, n = it / kStages;
                 // the consumers must have released the stage's previous use
                 if (n > 0 && !mbar_wait_bounded(empty + s, (n - 1) & 1, stop, kWaitLimit)) { ok = false; break; }
                 unsigned char* st = smem + s * L::kStage;
-                const int e = j * kTile;
+                const int e = j * L::kElems;
                 mbar_expect_tx(full + s, L::kStage);
                 unsigned o = 0;
                 if (!DEFER) { bulk_load(st, U.t1 + e, L::kF, full + s); o += L::kF; }
@@ -180,7 +186,7 @@ fused_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restri
     unsigned it = 0;
     for (long long c = blockIdx.x; c < num_chunks; c += gridDim.x) {
         FusedUnit<G> U;
-        if (!fused_resolve<ADAMW, G, DEFER>(c, descs, chunks, flat, p, U)) continue;
+        if (!fused_resolve<ADAMW, G, DEFER>(c, descs, chunks, flat, p, L::kElems, U)) continue;
         if (!U.vec) {                                   // misaligned tensor: scalar path, no staging
             for (int e = threadIdx.x; e < U.len; e += kThreads) {
                 float mm = ADAMW ? U.m[e] : 0.0f, vv = ADAMW ? U.v[e] : 0.0f;
@@ -201,7 +207,9 @@ fused_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restri
                 return;
             }
             const unsigned char* st = smem + s * L::kStage;
-            const int tt = threadIdx.x * 8;
+#pragma unroll 1
+            for (int h = 0; h < L::kMult; ++h) {
+            const int tt = (h * kThreads + threadIdx.x) * 8;
             unsigned o = 0;
             FVec<8> a1, a0, mm, vv;
             if (!DEFER) { a1 = lds_f8(reinterpret_cast<const float*>(st) + tt); o += L::kF; }
@@ -212,7 +220,7 @@ fused_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restri
             }
             FVec<8> b0 = scaled<8>(lds_g8(reinterpret_cast<const G*>(st + o) + tt), gs0); o += L::kGb;
             FVec<8> b1 = scaled<8>(lds_g8(reinterpret_cast<const G*>(st + o) + tt), gs1);
-            const int e = j * kTile + tt;
+            const int e = j * L::kElems + tt;
             if (DEFER) {
                 a1 = a0;
                 optim_step_vec<ADAMW, 8>(a1, mm, vv, b0, p.step0);
@@ -222,13 +230,14 @@ fused_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restri
             st_f(U.out + e, a1);
             if (U.wb) st_bf16(U.wb + e, a1);
             if (ADAMW) { st_f(U.m + e, mm); st_f(U.v + e, vv); }
+            }
             // Hand the stage back only now: every lane's stores depend on what it read from
             // the stage, so by this point the shared-memory reads have certainly completed.
             __syncwarp();
             if (lane == 0) mbar_arrive(empty + s);
         }
-        // ragged rest of the chunk (less than one tile): register path
-        const int done = U.full_tiles * kTile;
+        // ragged rest of the chunk (less than one stage): register path
+        const int done = U.full_tiles * L::kElems;
         if (done < U.len)
             fused_chunk_vec<ADAMW, G, 8, DEFER, false>(U.out + done, U.t1 + done, U.t0 + done,
                                                        ADAMW ? U.m + done : nullptr, ADAMW ? U.v + done : nullptr,
