@@ -69,6 +69,7 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-params", type=int, default=1 << 26)
+    ap.add_argument("--e2e-staging", type=int, default=1 << 23, help="parameters per staged piece in the e2e leg")
     ap.add_argument("--cpu-params", type=int, default=1 << 24)
     return ap.parse_args()
 
@@ -479,7 +480,7 @@ def run_e2e(torch, b, args, cfg, opt):
             torch.cuda.synchronize()
             l0 = ctx.launch_count()
             t0 = time.perf_counter()
-        ctx.step_host(t, staging_elems=1 << 23, allow_nonfinite=True)
+        ctx.step_host(t, staging_elems=args.e2e_staging, allow_nonfinite=True)
     torch.cuda.synchronize()
     dt = (time.perf_counter() - t0) / 3
     launches = (ctx.launch_count() - l0) // 3
@@ -487,7 +488,7 @@ def run_e2e(torch, b, args, cfg, opt):
     return {"value": n / dt, "unit": UNIT, "h2d_bytes_per_step": 18 * n, "d2h_bytes_per_step": 12 * n + 64,
             "ms_per_step": dt * 1e3, "gpu_launches_per_step": launches,
             "sample": f"{n}-parameter flat slice; theta, m, v, g0, g1, g_slow in pinned host memory, "
-                      f"streamed through gxpo_step_host in 8388608-parameter pieces"}
+                      f"streamed through gxpo_step_host in {args.e2e_staging}-parameter pieces"}
 
 
 def run_surrogate(args):
