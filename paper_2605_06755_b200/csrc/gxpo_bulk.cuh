@@ -22,7 +22,7 @@ namespace gxpo {
 constexpr int kMaxStages = 3;
 constexpr int kConsumerWarps = kThreads / 32;
 constexpr int kBulkThreads = kThreads + 32;         // consumers + one producer warp
-constexpr unsigned kWaitLimit = 1u << 22;           // polls per wait (each poll may itself block briefly)
+constexpr unsigned kWaitLimit = 1u << 20;           // polls per wait (each poll may itself block briefly)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
