@@ -3,7 +3,7 @@
 // one would expect to win on this GPU and the measurement says otherwise.
 //
 // One producer thread streams whole stages (one or two 2048-element tiles of every input
-// array) into a shared-memory ring with cp.async.bulk (no tensor map, no multicast, this GPU's own
+// array) into a shared-memory ring with cp.async.bulk (plain 1-D copies to this CTA only, from this GPU's own
 // memory only); eight consumer warps pick a tile up when its mbarrier completes, do the
 // same per-coordinate arithmetic as the register-staged kernel (same functions, hence the
 // same bits) and store straight from registers.  All but one stage of the ring are in flight
