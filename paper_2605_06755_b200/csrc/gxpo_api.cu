@@ -19,8 +19,8 @@ namespace {
 constexpr int kDefaultCtasStep = 2;    // measured best for the 14R/12W sweep
 constexpr int kDefaultCtasStepLight = 3;  // 14R/4W (deferred first probe): read-heavy, wants more loads in flight
 constexpr int kDefaultCtasExtrap = 4;  // the extrapolation needs more warps to cover its arithmetic
-constexpr int kDefaultCtasFused = 3;
-constexpr int kDefaultCtasBulk = 1;    // one CTA per SM with a 3-stage ring measured best (2 is as good, 4+ stages worse)
+constexpr int kDefaultCtasFused = 3;   // register-staged fused sweep (its 118-120 registers allow 2)
+constexpr int kDefaultCtasBulk = 1;    // bulk-copy staged fused sweep: one ring per SM (two measure the same)
 
 enum Phase { IDLE = 0, PROBED0 = 1, PROBED1 = 2, EXTRAPOLATED = 3, SLOW_DONE = 4, PROBED0_DEFERRED = 5 };
 
