@@ -38,3 +38,27 @@ def test_status_strings_and_defaults_need_no_gpu():
     assert abs(cfg.alpha - 0.5) < 1e-7 and abs(cfg.tau - 0.5) < 1e-15 and abs(cfg.delta - 1e-8) < 1e-12
     assert opt.kind == b.OPT_ADAMW and opt.lr == 1e-7 and opt.beta2 == 0.999
     assert b._lib.gxpo_status_string(b.ERR_STATE).decode() == "call out of order"
+
+
+def test_header_is_c99_and_a_plain_c_program_links_against_the_library(tmp_path):
+    """The boundary is a C ABI: include/gxpo.h must compile as C99 and a C program must
+    link against libgxpo.so and call it without any Python in between."""
+    import subprocess
+    from paper_2605_06755_b200 import build
+    lib = build.build_library()
+    src = tmp_path / "use.c"
+    src.write_text(
+        '#include <stdio.h>\n#include <string.h>\n#include "gxpo.h"\n'
+        "int main(void) {\n"
+        "    gxpo_cfg c; gxpo_opt_cfg o;\n"
+        "    gxpo_default_cfg(&c, &o);\n"
+        "    if (c.K != 5 || o.kind != GXPO_OPT_ADAMW) return 2;\n"
+        '    if (strcmp(gxpo_status_string(GXPO_ERR_TIMEOUT), "device-side wait timed out") != 0) return 3;\n'
+        "    if (gxpo_probe_step(NULL, 0, NULL) != GXPO_ERR_INVALID_ARG) return 4;\n"
+        '    printf("%d %lld\\n", c.window, (long long)GXPO_NOALLOC_MAX_PARAMS);\n'
+        "    return 0;\n}\n")
+    exe = tmp_path / "use"
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-I", os.path.join(ROOT, "include"),
+                           str(src), "-o", str(exe), lib, "-Wl,-rpath," + os.path.dirname(lib)])
+    out = subprocess.check_output([str(exe)]).decode().split()
+    assert out == ["20", "2147483648"]
