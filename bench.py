@@ -404,6 +404,8 @@ def run_ours(args):
     if args.variant == 3 or (args.variant == 0 and n_chunks >= 32 * props.multi_processor_count):
         # the fused sweep runs in its bulk-copy staged kernel (the library's default for long lists)
         kernel_of["probe_extrapolate"] = kernel_of["probe_extrapolate_deferred"] = "fused_bulk_kernel"
+        for nm in ("probe_step0", "probe_step1", "slow_step", "fallback_step"):   # AdamW sweeps that write m, v back
+            kernel_of[nm] = "step_bulk_kernel"
     kernels = {nm: {"kernel": kernel_of[nm], "ms": ms, "bytes_per_param": alg_bytes[nm],
                     "gbs": alg_bytes[nm] * d / (ms * 1e-3) / 1e9} for nm, ms in per.items()}
     # dominant kernel = the kernel function with the largest share of the step; its figures

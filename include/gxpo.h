@@ -316,11 +316,11 @@ gxpo_status gxpo_step_host(gxpo_ctx* ctx, const gxpo_tensor* list, int count,
                            long long staging_elems, void* stream, gxpo_gate_result* out);
 
 /* Launch-shape knobs, for benchmarking: resident CTAs per SM (0 = default), the
- * memory-access variant (0 = default: 256-bit loads and, for gxpo_probe_extrapolate on
- * lists of at least 32 chunks per SM, a producer thread that stages whole tiles in shared
- * memory with bulk asynchronous copies; 1 = 128-bit loads, register staging everywhere;
- * 2 = 256-bit loads, register staging everywhere; 3 = like 0 for lists of any length)
- * and the
+ * memory-access variant (0 = default: 256-bit loads; on lists of at least 32 chunks per SM
+ * the fused sweep and the AdamW sweeps that write m and v back are fed by a producer thread
+ * that stages whole tiles in shared memory with bulk asynchronous copies; 1 = 128-bit
+ * loads, register staging everywhere; 2 = 256-bit loads, register staging everywhere;
+ * 3 = like 0 for lists of any length) and the
  * number of 2048-element tiles a CTA takes per round-robin turn (0 = default: 16, or
  * 8 / 4 for lists of only a few thousand 32768-element chunks; else 1, 2, 4, 8 or 16).  Element-wise results are identical across all settings; only the
  * summation order of the norm changes. */

@@ -241,6 +241,38 @@ FusedFn pick_fused(bool adamw, bool bf16, int variant, bool defer, bool diag) {
     return defer ? pick_fused_t<true, false>(adamw, bf16, variant) : pick_fused_t<false, false>(adamw, bf16, variant);
 }
 
+// The bulk-copy staged AdamW sweep: one CTA per SM, whole chunks.
+typedef void (*StepBulkFn)(const TensorDesc*, const ChunkRef*, long long, TensorDesc, StepParams, double*,
+                           unsigned*, double*, int*);
+template <typename G>
+gxpo_status launch_step_bulk_t(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
+                               long long num_chunks, const TensorDesc& flat, const StepParams& p, double* sumsq) {
+    StepBulkFn fn = step_bulk_kernel<true, G>;
+    const int smem = (int)StepLayout<true, G>::kTotal;
+    int resident = 0;
+    for (int i = 0; i < c->occ_n; ++i)
+        if (c->occ_key[i] == (const void*)fn) resident = c->occ_val[i];
+    if (resident == 0) {
+        CUDA_TRY(c, cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, (const void*)fn, kBulkThreads, (size_t)smem) != cudaSuccess || resident < 1)
+            resident = 1;
+        if (c->occ_n < 32) { c->occ_key[c->occ_n] = (const void*)fn; c->occ_val[c->occ_n] = resident; c->occ_n += 1; }
+    }
+    int per_sm = c->ctas_per_sm > 0 ? c->ctas_per_sm : kDefaultCtasBulk;
+    if (per_sm > resident) per_sm = resident;
+    long long g = (long long)c->sm_count * per_sm;
+    if (g > num_chunks) g = num_chunks;
+    fn<<<(int)g, kBulkThreads, smem, s>>>(descs, chunks, num_chunks, flat, p, c->d_partials, c->d_ticket, sumsq, c->d_err);
+    c->launches += 1;
+    CUDA_TRY(c, cudaGetLastError());
+    return GXPO_OK;
+}
+gxpo_status launch_step_bulk(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
+                             long long num_chunks, const TensorDesc& flat, const StepParams& p, double* sumsq) {
+    return c->grad_dtype == GXPO_BF16 ? launch_step_bulk_t<uint16_t>(c, s, descs, chunks, num_chunks, flat, p, sumsq)
+                                      : launch_step_bulk_t<float>(c, s, descs, chunks, num_chunks, flat, p, sumsq);
+}
+
 // Launch one OptimStep sweep over either the bound list (chunks != null) or one
 // flat piece described by `flat`.
 gxpo_status launch_step(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
@@ -251,6 +283,10 @@ gxpo_status launch_step(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, co
         return GXPO_OK;
     }
     const bool adamw = c->opt.kind == GXPO_OPT_ADAMW;
+    // AdamW sweeps that write m and v back run bulk-copy staged on long lists (default) or
+    // always (variant 3); the read-heavy deferred probe and plain GD stay register-staged.
+    if (adamw && p.write_state && ((c->variant == 0 && num_chunks >= 32LL * c->sm_count) || c->variant == 3))
+        return launch_step_bulk(c, s, descs, chunks, num_chunks, flat, p, sumsq);
     StepFn fn = pick_step(adamw, c->grad_dtype == GXPO_BF16, c->variant);
     const int ush = unit_shift_for(c, num_chunks);
     const int grid = grid_for(c, (const void*)fn, num_chunks << ush,

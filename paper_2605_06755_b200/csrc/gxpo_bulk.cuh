@@ -246,6 +246,159 @@ fused_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restri
     }
 }
 
+// ---------------------------------------------------------------------------
+// The AdamW sweep with the same staging, for the calls that write m and v back (slow
+// step, fallback step, non-deferred probe steps): 14 R + 12 W per parameter.  Measured on a
+// 7.6e9-parameter list: two stages of 4096 elements 6.55 TB/s against 6.43 register-staged
+// (three stages of 2048: 6.34; two of 8192: 6.04).  The read-heavy deferred probe (14 R +
+// 4 W) is slower staged (5.8 against 6.8 TB/s) and stays register-staged.  Consumers
+// accumulate sum(g^2) like the register-staged kernel and reduce it among themselves on a
+// named barrier (the producer warp has left by then).
+// ---------------------------------------------------------------------------
+constexpr int kStepMult = 2;       // tiles per stage
+constexpr int kStepStages = 2;
+template <bool ADAMW, typename G>
+struct StepLayout {
+    static constexpr int kElems = kTile * kStepMult;
+    static constexpr unsigned kF = kElems * sizeof(float);
+    static constexpr unsigned kGb = kElems * sizeof(G);
+    static constexpr unsigned kStage = (ADAMW ? 3 : 1) * kF + kGb;
+    static constexpr unsigned kTotal = kStepStages * kStage + 2 * kMaxStages * sizeof(uint64_t) + 16;
+};
+template <typename G> struct StepUnit {
+    const float* in; float* out; float* snap; float* m; float* v; const G* g; uint16_t* wb;
+    int len, full_tiles; bool vec;
+};
+template <bool ADAMW, typename G>
+__device__ __forceinline__ bool step_resolve(long long c, const TensorDesc* descs, const ChunkRef* chunks,
+                                             const TensorDesc& flat, const StepParams& p, int stage_elems, StepUnit<G>& U) {
+    ChunkRef ref; TensorDesc d;
+    if (chunks) { ref = chunks[c]; d = descs[ref.tensor]; } else { ref.tensor = 0; ref.chunk = (unsigned)c; d = flat; }
+    const long long off = (long long)ref.chunk * kChunk;
+    const long long rem = d.n - off;
+    U.len = 0; U.full_tiles = 0; U.vec = false;
+    if (rem <= 0) return false;
+    U.len = rem < kChunk ? (int)rem : kChunk;
+    U.in = (p.in_sel ? d.work : d.theta) + off;
+    U.out = (p.out_sel ? d.work : d.theta) + off;
+    U.snap = p.snapshot ? d.work + off : nullptr;
+    U.m = ADAMW ? d.m + off : nullptr; U.v = ADAMW ? d.v + off : nullptr;
+    const void* gsel = p.which_grad == 0 ? d.g[0] : (p.which_grad == 1 ? d.g[1] : d.g[2]);
+    U.g = reinterpret_cast<const G*>(gsel) + off;
+    U.wb = (p.emit && d.wb) ? d.wb + off : nullptr;
+    U.vec = aligned32(U.in) && aligned32(U.out) && aligned32(U.g) && (!ADAMW || (aligned32(U.m) && aligned32(U.v))) &&
+            (!p.snapshot || aligned32(U.snap)) && aligned16(U.wb);
+    U.full_tiles = U.vec ? U.len / stage_elems : 0;
+    return true;
+}
+__device__ __forceinline__ double consumer_sum(double x, double* smem8) {
+    x = warp_sum(x);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    asm volatile("bar.sync 1, %0;" :: "r"(kThreads) : "memory");
+    if (lane == 0) smem8[warp] = x;
+    asm volatile("bar.sync 1, %0;" :: "r"(kThreads) : "memory");
+    double t = 0.0;
+    if (warp == 0) { t = (lane < kConsumerWarps) ? smem8[lane] : 0.0; t = warp_sum(t); }
+    return t;
+}
+template <bool ADAMW, typename G>
+__global__ void __launch_bounds__(kBulkThreads, 1)
+step_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restrict__ chunks,
+                 long long num_chunks, TensorDesc flat, StepParams p, double* partials, unsigned* ticket,
+                 double* sumsq_out, int* error_word) {
+    typedef StepLayout<ADAMW, G> L;
+    constexpr int kStages = kStepStages;
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ double red[8];
+    __shared__ bool is_last;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStages * L::kStage);
+    uint64_t* empty = full + kMaxStages;
+    volatile int* stop = reinterpret_cast<volatile int*>(empty + kMaxStages);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, kConsumerWarps); }
+        *stop = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (warp == kConsumerWarps) {
+        if (lane != 0) return;
+        unsigned it = 0; bool ok = true;
+        for (long long c = blockIdx.x; c < num_chunks && ok; c += gridDim.x) {
+            StepUnit<G> U;
+            if (!step_resolve<ADAMW, G>(c, descs, chunks, flat, p, L::kElems, U)) continue;
+            for (int j = 0; j < U.full_tiles; ++j, ++it) {
+                const unsigned s = it % kStages, n = it / kStages;
+                if (n > 0 && !mbar_wait_bounded(empty + s, (n - 1) & 1, stop, kWaitLimit)) { ok = false; break; }
+                unsigned char* st = smem + s * L::kStage;
+                const int e = j * L::kElems;
+                mbar_expect_tx(full + s, L::kStage);
+                unsigned o = 0;
+                bulk_load(st, U.in + e, L::kF, full + s); o += L::kF;
+                if (ADAMW) { bulk_load(st + o, U.m + e, L::kF, full + s); o += L::kF; bulk_load(st + o, U.v + e, L::kF, full + s); o += L::kF; }
+                bulk_load(st + o, U.g + e, L::kGb, full + s);
+            }
+        }
+        if (!ok) {
+            *stop = 1; atomicExch(error_word, 1);
+            for (unsigned k = 0; k < (unsigned)kStages && k < it; ++k) {
+                const unsigned i2 = it - 1 - k;
+                for (unsigned w = 0; w < kWaitLimit && !mbar_try_wait(full + i2 % kStages, (i2 / kStages) & 1); ++w) __nanosleep(64);
+            }
+        }
+        return;
+    }
+    const float gscale = p.gscale ? __ldg(p.gscale) : 1.0f;
+    double acc = 0.0; unsigned it = 0; bool alive = true;
+    for (long long c = blockIdx.x; c < num_chunks && alive; c += gridDim.x) {
+        StepUnit<G> U;
+        if (!step_resolve<ADAMW, G>(c, descs, chunks, flat, p, L::kElems, U)) continue;
+        if (!U.vec) { step_chunk_scalar<ADAMW, G>(U.out, U.in, U.snap, U.m, U.v, U.g, U.len, p, gscale, acc, U.wb); continue; }
+        for (int j = 0; j < U.full_tiles; ++j, ++it) {
+            const unsigned s = it % kStages, n = it / kStages;
+            if (!mbar_wait_bounded(full + s, n & 1, stop, kWaitLimit)) { *stop = 1; atomicExch(error_word, 1); alive = false; break; }
+            const unsigned char* st = smem + s * L::kStage;
+#pragma unroll 1
+            for (int h = 0; h < kStepMult; ++h) {
+                const int tt = (h * kThreads + threadIdx.x) * 8;
+                unsigned o = 0;
+                FVec<8> th, mm, vv;
+                th = lds_f8(reinterpret_cast<const float*>(st) + tt); o += L::kF;
+                if (ADAMW) { mm = lds_f8(reinterpret_cast<const float*>(st + o) + tt); o += L::kF; vv = lds_f8(reinterpret_cast<const float*>(st + o) + tt); o += L::kF; }
+                const FVec<8> gg = lds_g8(reinterpret_cast<const G*>(st + o) + tt);
+                const int e = j * L::kElems + tt;
+                if (U.snap) st_f(U.snap + e, th);
+                float sq = 0.0f;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) { sq = fmaf(gg.x[i], gg.x[i], sq); optim_step_elem<ADAMW>(th.x[i], mm.x[i], vv.x[i], __fmul_rn(gg.x[i], gscale), p); }
+                if (!p.skip_out) st_f(U.out + e, th);
+                if (U.wb) st_bf16(U.wb + e, th);
+                if (ADAMW && p.write_state) { st_f(U.m + e, mm); st_f(U.v + e, vv); }
+                acc += (double)sq;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty + s);
+        }
+        if (!alive) break;
+        const int done = U.full_tiles * L::kElems;
+        if (done < U.len)
+            step_chunk_vec<ADAMW, G, 8>(U.out + done, U.in + done, U.snap ? U.snap + done : nullptr, ADAMW ? U.m + done : nullptr,
+                                        ADAMW ? U.v + done : nullptr, U.g + done, U.len - done, p, gscale, acc, U.wb ? U.wb + done : nullptr);
+    }
+    if (p.want_norm) {
+        const double tot = consumer_sum(acc, red);
+        if (threadIdx.x == 0) { partials[blockIdx.x] = tot; __threadfence(); is_last = (atomicAdd(ticket, 1u) == gridDim.x - 1); }
+        asm volatile("bar.sync 1, %0;" :: "r"(kThreads) : "memory");
+        if (is_last) {
+            __threadfence();
+            double sum = 0.0;
+            for (unsigned i = threadIdx.x; i < gridDim.x; i += kThreads) sum += __ldcg(partials + i);
+            sum = consumer_sum(sum, red);
+            if (threadIdx.x == 0) { *sumsq_out = sum; *ticket = 0u; }
+        }
+    }
+}
+
 // Nothing ever completes the barrier this kernel waits on: the bounded wait has to give up
 // after `limit` polls and raise the error word.  Used to check that path end to end.
 __global__ void bounded_wait_probe_kernel(unsigned limit, int* error_word) {
