@@ -66,6 +66,8 @@ def parse_args():
     ap.add_argument("--emit-bf16", action="store_true",
                     help="also keep bfloat16 model-weight copies (gxpo_bind_model_weights, bf16-only theta1): "
                          "16 + 30 + 28 = 74 B/param, and the caller needs no cast sweeps")
+    ap.add_argument("--diagnostics", action="store_true",
+                    help="gather the per-step diagnostics too (adds a 4 B/param <g0, g_slow> pass after the slow step)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-params", type=int, default=1 << 26)
@@ -308,6 +310,8 @@ def run_ours(args):
     ctx = b.Context(cfg, opt, b.BF16)
     ctx.tune(args.ctas, args.variant, args.unit_tiles)
     ctx.bind(ptrs)
+    diag = bool(getattr(args, "diagnostics", False)) and not args.fallback
+    ctx.enable_diagnostics(diag)
     if emit:
         weights = torch.empty(d, dtype=torch.bfloat16, device="cuda")
         offs, acc = [], 0
@@ -399,6 +403,8 @@ def run_ours(args):
         alg_bytes["probe_step0_deferred"] -= 2
         alg_bytes["probe_extrapolate_deferred"] += 2
         alg_bytes["slow_step"] += 2
+    if diag and not alias:      # <g0, g_slow>: one more read of both gradients, timed with the slow step
+        alg_bytes["slow_step"] += 4
     kernel_of = dict(KERNEL_OF)
     n_chunks = sum((k + 32767) // 32768 for _, k in shapes)
     if args.variant == 3 or (args.variant == 0 and n_chunks >= 32 * props.multi_processor_count):
@@ -439,7 +445,7 @@ def run_ours(args):
                    {"deferred": "active (probe with deferred state, probe+extrapolate in one sweep, slow step, gate)",
                     "fused": "active (probe, probe+extrapolate in one sweep, slow step, gate)",
                     "unfused": "active (probe, probe, extrapolate, slow step, gate)"}[flow],
-                   "bf16_model_weight_copies": emit, "g_slow_aliases_g0": alias, "l2": "inputs larger than L2 (no flush needed)",
+                   "bf16_model_weight_copies": emit, "diagnostics": diag, "g_slow_aliases_g0": alias, "l2": "inputs larger than L2 (no flush needed)",
                    "parallelism": f"dp{world} (independent shards, one 8-byte all-reduce per step)" if world > 1 else "1 GPU"},
         "hbm_gbs_whole_step": whole_gbs, "hbm_frac_whole_step": whole_gbs / peak,
         "hbm_frac_of_8tbs_nominal": whole_gbs / 8000.0,

@@ -270,6 +270,11 @@ gxpo_status gxpo_clip_grad_norm(gxpo_ctx* ctx, int which, double max_norm, void*
  *   inactive_frac                : 1 - |A_t| / n
  * A coordinate whose ratio or scale is not a finite float32 is "irregular": it is
  * counted in n_irregular and left out of the ratio, scale and displacement figures.
+ * Accuracy: the counts are exact; the sums are float64 sums of float32 partial sums over
+ * 8 consecutive coordinates, so a figure built from non-negative terms (the norms,
+ * disp_ratio) is within 3e-7 relative of the exact one, and a term whose square is under
+ * float32's normal range (|x| < 1e-19) may be lost; groups whose float32 partial sum
+ * would exceed 1e30 are summed in float64 throughout.
  * With a caller-owned sum-of-squares buffer (gxpo_set_sumsq_buffer) gslow_norm and the
  * cosine use whatever that buffer holds; everything else is this context's share. */
 typedef struct {

@@ -313,11 +313,12 @@ gxpo_status launch_extrap(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, 
 }
 
 // The bulk-copy staged variant of the fused sweep: one CTA per SM, whole chunks.
-typedef void (*BulkFn)(const TensorDesc*, const ChunkRef*, long long, TensorDesc, FusedParams, int*);
+typedef void (*BulkFn)(const TensorDesc*, const ChunkRef*, long long, TensorDesc, FusedParams, int*, double*,
+                       unsigned*, double*);
 template <bool ADAMW, typename G, bool DEFER>
 gxpo_status launch_bulk_t(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
-                          long long num_chunks, const TensorDesc& flat, const FusedParams& p) {
-    BulkFn fn = fused_bulk_kernel<ADAMW, G, DEFER>;
+                          long long num_chunks, const TensorDesc& flat, const FusedParams& p, bool diag) {
+    BulkFn fn = diag ? fused_bulk_kernel<ADAMW, G, DEFER, true> : fused_bulk_kernel<ADAMW, G, DEFER, false>;
     const int smem = (int)BulkLayout<ADAMW, G, DEFER>::kTotal;
     // first launch of this instantiation in this context: allow the ring's shared memory and
     // find out how many CTAs fit; remembered in the occupancy cache afterwards
@@ -334,16 +335,18 @@ gxpo_status launch_bulk_t(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, 
     if (per_sm > resident) per_sm = resident;
     long long g = (long long)c->sm_count * per_sm;
     if (g > num_chunks) g = num_chunks;
-    fn<<<(int)g, kBulkThreads, smem, s>>>(descs, chunks, num_chunks, flat, p, c->d_err);
+    fn<<<(int)g, kBulkThreads, smem, s>>>(descs, chunks, num_chunks, flat, p, c->d_err, c->d_diag_partials,
+                                          c->d_ticket, c->d_diag);
     c->launches += 1;
     CUDA_TRY(c, cudaGetLastError());
     return GXPO_OK;
 }
 gxpo_status launch_fused_bulk(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
-                              long long num_chunks, const TensorDesc& flat, const FusedParams& p, bool defer) {
+                              long long num_chunks, const TensorDesc& flat, const FusedParams& p, bool defer,
+                              bool diag) {
     const bool adamw = c->opt.kind == GXPO_OPT_ADAMW, bf16 = c->grad_dtype == GXPO_BF16;
-#define GXPO_BULK(A, G) (defer ? launch_bulk_t<A, G, true>(c, s, descs, chunks, num_chunks, flat, p) \
-                               : launch_bulk_t<A, G, false>(c, s, descs, chunks, num_chunks, flat, p))
+#define GXPO_BULK(A, G) (defer ? launch_bulk_t<A, G, true>(c, s, descs, chunks, num_chunks, flat, p, diag) \
+                               : launch_bulk_t<A, G, false>(c, s, descs, chunks, num_chunks, flat, p, diag))
     if (adamw) return bf16 ? GXPO_BULK(true, uint16_t) : GXPO_BULK(true, float);
     return bf16 ? GXPO_BULK(false, uint16_t) : GXPO_BULK(false, float);
 #undef GXPO_BULK
@@ -358,11 +361,10 @@ gxpo_status launch_fused(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, c
     }
     // default (0): the bulk-copy staged kernel for lists long enough to keep every SM's ring
     // busy (it deals whole chunks, one CTA per SM), register staging for short lists; 3
-    // forces bulk staging, 1 and 2 force register staging.  Diagnostics exist only in the
-    // register-staged kernel.
+    // forces bulk staging, 1 and 2 force register staging.
     const bool long_list = num_chunks >= 32LL * c->sm_count;
-    if (((c->variant == 0 && long_list) || c->variant == 3) && !diag)
-        return launch_fused_bulk(c, s, descs, chunks, num_chunks, flat, p, defer);
+    if ((c->variant == 0 && long_list) || c->variant == 3)
+        return launch_fused_bulk(c, s, descs, chunks, num_chunks, flat, p, defer, diag);
     FusedFn fn = pick_fused(c->opt.kind == GXPO_OPT_ADAMW, c->grad_dtype == GXPO_BF16, c->variant == 1 ? 1 : 2, defer, diag);
     const int ush = unit_shift_for(c, num_chunks);
     const int grid = grid_for(c, (const void*)fn, num_chunks << ush, kDefaultCtasFused);

@@ -108,6 +108,18 @@ __device__ __forceinline__ bool fused_resolve(long long c, const TensorDesc* des
     return true;
 }
 
+// sum over the 256 consumer threads on named barrier 1 (the producer warp takes no part);
+// valid in thread 0
+__device__ __forceinline__ double consumer_sum(double x, double* smem8) {
+    x = warp_sum(x);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    asm volatile("bar.sync 1, %0;" :: "r"(kThreads) : "memory");
+    if (lane == 0) smem8[warp] = x;
+    asm volatile("bar.sync 1, %0;" :: "r"(kThreads) : "memory");
+    double t = 0.0;
+    if (warp == 0) { t = (lane < kConsumerWarps) ? smem8[lane] : 0.0; t = warp_sum(t); }
+    return t;
+}
 // Shared memory per stage: [theta1 unless DEFER] theta0 [m v if ADAMW] g0 g1, kMult tiles each.
 // Ring shape, measured on a 7.6e9-parameter list: what matters is about 64 KB in flight per SM
 // in as few, as large pieces as possible.  Deferred sweep (5 arrays): 2 stages of 4096
@@ -124,10 +136,11 @@ struct BulkLayout {
     static constexpr unsigned kTotal = kStagesN * kStage + 2 * kMaxStages * sizeof(uint64_t) + 16;
 };
 
-template <bool ADAMW, typename G, bool DEFER>
+template <bool ADAMW, typename G, bool DEFER, bool DIAG>
 __global__ void __launch_bounds__(kBulkThreads, 1)
 fused_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restrict__ chunks,
-                  long long num_chunks, TensorDesc flat, FusedParams p, int* error_word) {
+                  long long num_chunks, TensorDesc flat, FusedParams p, int* error_word,
+                  double* diag_partials, unsigned* ticket, double* diag_out) {
     typedef BulkLayout<ADAMW, G, DEFER> L;
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int kStages = L::kStagesN;
@@ -182,17 +195,25 @@ fused_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restri
     }
 
     // ---- consumers
+    __shared__ double red[8];
+    __shared__ bool is_last;
+    DiagAcc acc;
+    if (DIAG) {
+#pragma unroll
+        for (int q = 0; q < kDiagN; ++q) acc.v[q] = 0.0;
+    }
+    bool alive = true;
     const float gs0 = p.ex.gscale0 ? __ldg(p.ex.gscale0) : 1.0f, gs1 = p.ex.gscale1 ? __ldg(p.ex.gscale1) : 1.0f;
     unsigned it = 0;
-    for (long long c = blockIdx.x; c < num_chunks; c += gridDim.x) {
+    for (long long c = blockIdx.x; c < num_chunks && alive; c += gridDim.x) {
         FusedUnit<G> U;
         if (!fused_resolve<ADAMW, G, DEFER>(c, descs, chunks, flat, p, L::kElems, U)) continue;
         if (!U.vec) {                                   // misaligned tensor: scalar path, no staging
             for (int e = threadIdx.x; e < U.len; e += kThreads) {
                 float mm = ADAMW ? U.m[e] : 0.0f, vv = ADAMW ? U.v[e] : 0.0f;
-                const float x = fused_elem<ADAMW, DEFER, false>(DEFER ? 0.0f : U.t1[e], U.t0[e], mm, vv,
+                const float x = fused_elem<ADAMW, DEFER, DIAG>(DEFER ? 0.0f : U.t1[e], U.t0[e], mm, vv,
                                                                 __fmul_rn(ld_grad1(U.g0 + e), gs0),
-                                                                __fmul_rn(ld_grad1(U.g1 + e), gs1), p, nullptr);
+                                                                __fmul_rn(ld_grad1(U.g1 + e), gs1), p, &acc);
                 U.out[e] = x;
                 if (U.wb) U.wb[e] = to_bf16(x);
                 if (ADAMW) { U.m[e] = mm; U.v[e] = vv; }
@@ -204,7 +225,8 @@ fused_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restri
             if (!mbar_wait_bounded(full + s, n & 1, stop, kWaitLimit)) {
                 *stop = 1;
                 atomicExch(error_word, 1);
-                return;
+                alive = false;
+                break;
             }
             const unsigned char* st = smem + s * L::kStage;
 #pragma unroll 1
@@ -226,7 +248,7 @@ fused_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restri
                 optim_step_vec<ADAMW, 8>(a1, mm, vv, b0, p.step0);
             }
             optim_step_vec<ADAMW, 8>(a1, mm, vv, b1, p.step);
-            extrapolate_vec<8, false>(a1, a0, b0, b1, p.ex, nullptr);
+            extrapolate_vec<8, DIAG>(a1, a0, b0, b1, p.ex, &acc);
             st_f(U.out + e, a1);
             if (U.wb) st_bf16(U.wb + e, a1);
             if (ADAMW) { st_f(U.m + e, mm); st_f(U.v + e, vv); }
@@ -236,13 +258,38 @@ fused_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restri
             __syncwarp();
             if (lane == 0) mbar_arrive(empty + s);
         }
+        if (!alive) break;
         // ragged rest of the chunk (less than one stage): register path
         const int done = U.full_tiles * L::kElems;
         if (done < U.len)
-            fused_chunk_vec<ADAMW, G, 8, DEFER, false>(U.out + done, U.t1 + done, U.t0 + done,
+            fused_chunk_vec<ADAMW, G, 8, DEFER, DIAG>(U.out + done, U.t1 + done, U.t0 + done,
                                                        ADAMW ? U.m + done : nullptr, ADAMW ? U.v + done : nullptr,
-                                                       U.g0 + done, U.g1 + done, U.len - done, p, gs0, gs1, nullptr,
+                                                       U.g0 + done, U.g1 + done, U.len - done, p, gs0, gs1, &acc,
                                                        U.wb ? U.wb + done : nullptr);
+    }
+    if (DIAG) {
+        // every consumer thread gets here, also after a wait that gave up
+#pragma unroll
+        for (int q = 0; q < kDiagN; ++q) {
+            const double tot = consumer_sum(acc.v[q], red);
+            if (threadIdx.x == 0) diag_partials[q * kMaxGrid + blockIdx.x] = tot;
+        }
+        if (threadIdx.x == 0) {
+            __threadfence();
+            is_last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+        }
+        asm volatile("bar.sync 1, %0;" :: "r"(kThreads) : "memory");
+        if (is_last) {
+            __threadfence();
+#pragma unroll 1
+            for (int q = 0; q < kDiagN; ++q) {
+                double sum = 0.0;
+                for (unsigned i = threadIdx.x; i < gridDim.x; i += kThreads) sum += __ldcg(diag_partials + q * kMaxGrid + i);
+                sum = consumer_sum(sum, red);
+                if (threadIdx.x == 0) diag_out[q] = sum;
+            }
+            if (threadIdx.x == 0) *ticket = 0u;
+        }
     }
 }
 
@@ -290,16 +337,6 @@ __device__ __forceinline__ bool step_resolve(long long c, const TensorDesc* desc
             (!p.snapshot || aligned32(U.snap)) && aligned16(U.wb);
     U.full_tiles = U.vec ? U.len / stage_elems : 0;
     return true;
-}
-__device__ __forceinline__ double consumer_sum(double x, double* smem8) {
-    x = warp_sum(x);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    asm volatile("bar.sync 1, %0;" :: "r"(kThreads) : "memory");
-    if (lane == 0) smem8[warp] = x;
-    asm volatile("bar.sync 1, %0;" :: "r"(kThreads) : "memory");
-    double t = 0.0;
-    if (warp == 0) { t = (lane < kConsumerWarps) ? smem8[lane] : 0.0; t = warp_sum(t); }
-    return t;
 }
 template <bool ADAMW, typename G>
 __global__ void __launch_bounds__(kBulkThreads, 1)

@@ -60,12 +60,14 @@ def _oracle_diag(probs, gcfg, ocfg):
 @pytest.mark.parametrize("grad_dtype,kind,tame", [("bf16", "adamw", True), ("bf16", "adamw", False),
                                                    ("f32", "gd", True)])
 @pytest.mark.parametrize("K", [3, 5, 10])
-def test_diagnostics_match_the_oracle(flow, grad_dtype, kind, tame, K):
+@pytest.mark.parametrize("variant", [0, 3])            # 3: the shared-memory staged sweeps gather them too
+def test_diagnostics_match_the_oracle(flow, grad_dtype, kind, tame, K, variant):
     b = _binding()
     probs = _problems(grad_dtype, tame)
     cfg, opt = b.make_cfg(kind=b.OPT_ADAMW if kind == "adamw" else b.OPT_GD, lr=1e-3, K=K, alpha=0.5)
     ctx = b.Context(cfg, opt, b.BF16 if grad_dtype == "bf16" else b.F32)
     ctx.bind([p.ptrs() for p in probs])
+    ctx.tune(0, variant, 0)
     ctx.enable_diagnostics(True)
     gcfg, ocfg = gu.ora_cfgs(cfg, opt)
     want = _oracle_diag(probs, gcfg, ocfg)
@@ -99,7 +101,8 @@ def test_diagnostics_match_the_oracle(flow, grad_dtype, kind, tame, K):
     ctx.close()
 
 
-def test_switching_diagnostics_on_changes_no_output_and_call_order_is_checked():
+@pytest.mark.parametrize("variant", [0, 3])
+def test_switching_diagnostics_on_changes_no_output_and_call_order_is_checked(variant):
     b = _binding()
     outs = []
     for on in (False, True):
@@ -107,6 +110,7 @@ def test_switching_diagnostics_on_changes_no_output_and_call_order_is_checked():
         cfg, opt = b.make_cfg(lr=1e-3, K=5)
         ctx = b.Context(cfg, opt, b.BF16)
         ctx.bind([p.ptrs() for p in probs])
+        ctx.tune(0, variant, 0)
         with pytest.raises(b.GxpoError) as e:
             ctx.get_diagnostics()
         assert e.value.status == b.ERR_STATE
@@ -144,4 +148,96 @@ def test_cosine_is_nan_when_g_slow_shares_g0s_buffer():
     d = ctx.get_diagnostics()
     assert math.isnan(d.cos_g0_gslow)
     assert d.gslow_norm == pytest.approx(d.g0_norm, rel=1e-6)      # float32 partial sums inside the slow sweep
+    ctx.close()
+
+
+def test_long_list_diagnostics_in_the_default_launch_configuration():
+    """A flat list long enough that the default picks the shared-memory staged sweep
+    (200,000,003 parameters, ragged tail): the counts against a library count of
+    |g0| > delta, the norms against float64 library reductions, every figure against the
+    register-staged sweep's (whose figures the oracle checks above), and the outputs
+    bit for bit against a run with diagnostics off."""
+    import argparse
+    import gc
+
+    import torch
+
+    import bench
+    b = _binding()
+    runs = {}
+    for name, variant, on in (("staged", 0, True), ("registers", 2, True), ("plain", 0, False)):
+        gc.collect()
+        torch.cuda.empty_cache()
+        args = argparse.Namespace(workload="flat", layers=0, params=200_000_003)
+        free, _ = torch.cuda.mem_get_info()
+        shapes, desc, alias = bench.plan_workload(args, free)
+        d, ptrs, keep = bench.build_device_workload(torch, b, shapes, 77, alias)
+        assert d == 200_000_003
+        cfg, opt = b.make_cfg(lr=1e-3, K=5, alpha=0.5)
+        ctx = b.Context(cfg, opt, b.BF16)
+        ctx.bind(ptrs)
+        ctx.tune(0, variant, 0)
+        ctx.enable_diagnostics(on)
+        g0, g1 = keep[4], keep[5]
+        if name == "staged":
+            n_active = 0
+            sq0 = sq1 = 0.0
+            for s in range(0, d, 1 << 26):
+                a, c = g0[s:s + (1 << 26)].double(), g1[s:s + (1 << 26)].double()
+                n_active += int((a.abs() > cfg.delta).sum().item())
+                sq0 += float(torch.dot(a, a).item())
+                sq1 += float(torch.dot(c, c).item())
+                del a, c
+        res = ctx.active_step(allow_nonfinite=True, deferred=True)
+        diag = ctx.get_diagnostics() if on else None
+        runs[name] = (diag, res.norm, keep[0].clone(), keep[2].clone(), keep[3].clone())
+        ctx.close()
+        del keep, g0, g1
+    got, ref = runs["staged"][0], runs["registers"][0]
+    assert got.n == 200_000_003 and got.n_active == n_active
+    # a vector's 8 squares are added up in float32 before they reach the float64 sums
+    assert got.g0_norm == pytest.approx(math.sqrt(sq0), rel=1e-6)
+    assert got.g1_norm == pytest.approx(math.sqrt(sq1), rel=1e-6)
+    assert got.gslow_norm == pytest.approx(runs["staged"][1], rel=1e-12)
+    for k in ("n", "n_active", "n_irregular"):
+        assert getattr(got, k) == getattr(ref, k), k
+    # float64 sums of the same float32 terms, grouped by a different grid
+    for k in ("g0_norm", "g1_norm", "gslow_norm", "ratio_mean", "ratio_std", "scale_mean", "disp_ratio",
+              "cos_g0_gslow", "inactive_frac"):
+        assert getattr(got, k) == pytest.approx(getattr(ref, k), rel=1e-9), k
+    for i in (2, 3, 4):
+        assert torch.equal(runs["staged"][i], runs["plain"][i])
+        assert torch.equal(runs["staged"][i], runs["registers"][i])
+    assert runs["staged"][1] == runs["plain"][1]
+
+
+@pytest.mark.parametrize("variant", [0, 3])
+@pytest.mark.parametrize("K", [3, 5])
+def test_terms_beyond_float32_squares_are_summed_in_float64(K, variant):
+    """The vector paths pre-sum a vector's terms in float32 and must notice when that
+    would overflow: planted coordinates with r = 1e16 (r^2 = 1e32), g0 = 1e16 and
+    (d * scale)^2 far above 3e38 still give the oracle's float64 figures."""
+    b = _binding()
+    probs = _problems("f32", tame=True)
+    big = probs[0]
+    g0, g1 = big.np_in["g0"].copy(), big.np_in["g1"].copy()
+    for idx, a, c in ((100, 1e-3, 1e13), (8 * 4096 + 3, 1e16, 5e15), (70000, 1e-3, 2e13)):
+        g0[idx], g1[idx] = a, c
+    probs[0] = gu.Problem(big.np_in["theta"], big.np_in["m"], big.np_in["v"], g0, g1, big.np_in["gs"])
+    cfg, opt = b.make_cfg(kind=b.OPT_GD, lr=1e-3, K=K, alpha=0.5)
+    ctx = b.Context(cfg, opt, b.F32)
+    ctx.bind([p.ptrs() for p in probs])
+    ctx.tune(0, variant, 0)
+    ctx.enable_diagnostics(True)
+    gcfg, ocfg = gu.ora_cfgs(cfg, opt)
+    want = _oracle_diag(probs, gcfg, ocfg)
+    ctx.active_step(allow_nonfinite=True, deferred=True)
+    got = ctx.get_diagnostics()
+    assert got.n_active == want["n_active"] and got.n_irregular == want["n_irregular"]
+    assert want["g0_norm"] > 9e15                                       # the planted terms carry the sums
+    if K == 3:                                                           # (for K = 5 the scale of r = 1e16 is not a float32)
+        assert want["ratio_std"] > 1e12 and want["n_irregular"] == 0
+    for k in ("g0_norm", "g1_norm", "ratio_mean", "ratio_std", "scale_mean", "disp_ratio"):
+        assert math.isfinite(getattr(got, k)), k
+        assert getattr(got, k) == pytest.approx(want[k], rel=1e-5), k
     ctx.close()
