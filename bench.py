@@ -403,11 +403,12 @@ def run_ours(args):
         alg_bytes["probe_step0_deferred"] -= 2
         alg_bytes["probe_extrapolate_deferred"] += 2
         alg_bytes["slow_step"] += 2
-    if diag and not alias:      # <g0, g_slow>: one more read of both gradients, timed with the slow step
-        alg_bytes["slow_step"] += 4
     kernel_of = dict(KERNEL_OF)
     n_chunks = sum((k + 32767) // 32768 for _, k in shapes)
-    if args.variant == 3 or (args.variant == 0 and n_chunks >= 32 * props.multi_processor_count):
+    staged = args.variant == 3 or (args.variant == 0 and n_chunks >= 32 * props.multi_processor_count)
+    if diag and not alias:      # <g0, g_slow>, timed with the slow step: g0 read once more inside the staged
+        alg_bytes["slow_step"] += 2 if staged else 4      # sweep, else a pass of its own over both gradients
+    if staged:
         # the fused sweep runs in its bulk-copy staged kernel (the library's default for long lists)
         kernel_of["probe_extrapolate"] = kernel_of["probe_extrapolate_deferred"] = "fused_bulk_kernel"
         for nm in ("probe_step0", "probe_step1", "slow_step", "fallback_step"):   # AdamW sweeps that write m, v back

@@ -256,9 +256,11 @@ gxpo_status gxpo_clip_grad_norm(gxpo_ctx* ctx, int which, double max_norm, void*
 /* Per-step diagnostics of the active phase: the quantities the paper's appendix
  * tabulates ("Active-phase GXPO diagnostics").  Off by default.  When on, the sums are
  * gathered inside the extrapolation sweep (gxpo_extrapolate or gxpo_probe_extrapolate) at
- * no extra memory traffic; only <g0, g_slow> needs one more pass over the two gradient
- * buffers after the slow step (+4 bytes per parameter for bfloat16 gradients), and is
- * skipped (cos = NaN) when some tensor's g_slow shares g0's buffer.
+ * no extra memory traffic; only <g0, g_slow> needs g0 once more: the slow step's sweep
+ * reads it along (+2 bytes per parameter for bfloat16 gradients) where that sweep runs
+ * shared-memory staged (AdamW on long lists), otherwise one more pass over the two
+ * gradient buffers follows the slow step (+4 bytes per parameter).  It is skipped
+ * (cos = NaN) when some tensor's g_slow shares g0's buffer.
  *   g0_norm, g1_norm, gslow_norm : Euclidean norms over all coordinates
  *   cos_g0_gslow                 : <g0, g_slow> / (||g0|| ||g_slow||)
  *   ratio_mean, ratio_std        : mean and population standard deviation of the

@@ -243,12 +243,13 @@ FusedFn pick_fused(bool adamw, bool bf16, int variant, bool defer, bool diag) {
 
 // The bulk-copy staged AdamW sweep: one CTA per SM, whole chunks.
 typedef void (*StepBulkFn)(const TensorDesc*, const ChunkRef*, long long, TensorDesc, StepParams, double*,
-                           unsigned*, double*, int*);
+                           unsigned*, double*, int*, double*, double*);
 template <typename G>
 gxpo_status launch_step_bulk_t(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
-                               long long num_chunks, const TensorDesc& flat, const StepParams& p, double* sumsq) {
-    StepBulkFn fn = step_bulk_kernel<true, G>;
-    const int smem = (int)StepLayout<true, G>::kTotal;
+                               long long num_chunks, const TensorDesc& flat, const StepParams& p, double* sumsq,
+                               double* dot_out) {
+    StepBulkFn fn = dot_out ? step_bulk_kernel<true, G, true> : step_bulk_kernel<true, G, false>;
+    const int smem = dot_out ? (int)StepLayout<true, G, true>::kTotal : (int)StepLayout<true, G, false>::kTotal;
     int resident = 0;
     for (int i = 0; i < c->occ_n; ++i)
         if (c->occ_key[i] == (const void*)fn) resident = c->occ_val[i];
@@ -262,31 +263,41 @@ gxpo_status launch_step_bulk_t(gxpo_ctx* c, cudaStream_t s, const TensorDesc* de
     if (per_sm > resident) per_sm = resident;
     long long g = (long long)c->sm_count * per_sm;
     if (g > num_chunks) g = num_chunks;
-    fn<<<(int)g, kBulkThreads, smem, s>>>(descs, chunks, num_chunks, flat, p, c->d_partials, c->d_ticket, sumsq, c->d_err);
+    // the diagnostics' partial-sum array is idle between the extrapolation sweep and the next step
+    fn<<<(int)g, kBulkThreads, smem, s>>>(descs, chunks, num_chunks, flat, p, c->d_partials, c->d_ticket, sumsq, c->d_err,
+                                          c->d_diag_partials, dot_out);
     c->launches += 1;
     CUDA_TRY(c, cudaGetLastError());
     return GXPO_OK;
 }
 gxpo_status launch_step_bulk(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
-                             long long num_chunks, const TensorDesc& flat, const StepParams& p, double* sumsq) {
-    return c->grad_dtype == GXPO_BF16 ? launch_step_bulk_t<uint16_t>(c, s, descs, chunks, num_chunks, flat, p, sumsq)
-                                      : launch_step_bulk_t<float>(c, s, descs, chunks, num_chunks, flat, p, sumsq);
+                             long long num_chunks, const TensorDesc& flat, const StepParams& p, double* sumsq,
+                             double* dot_out) {
+    return c->grad_dtype == GXPO_BF16 ? launch_step_bulk_t<uint16_t>(c, s, descs, chunks, num_chunks, flat, p, sumsq, dot_out)
+                                      : launch_step_bulk_t<float>(c, s, descs, chunks, num_chunks, flat, p, sumsq, dot_out);
+}
+
+// AdamW sweeps that write m and v back run bulk-copy staged on long lists (default) or
+// always (variant 3); the read-heavy deferred probe and plain GD stay register-staged.
+bool step_runs_staged(const gxpo_ctx* c, const StepParams& p, long long num_chunks) {
+    return c->opt.kind == GXPO_OPT_ADAMW && p.write_state &&
+           ((c->variant == 0 && num_chunks >= 32LL * c->sm_count) || c->variant == 3);
 }
 
 // Launch one OptimStep sweep over either the bound list (chunks != null) or one
 // flat piece described by `flat`.
+// dot_out (only honoured when the sweep runs staged, see step_runs_staged; want_norm must be
+// set): also leave <g0, g> there.
 gxpo_status launch_step(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
                         long long num_chunks, const TensorDesc& flat, const StepParams& p,
-                        double* sumsq) {
+                        double* sumsq, double* dot_out = nullptr) {
     if (num_chunks <= 0) {
         if (p.want_norm) CUDA_TRY(c, cudaMemsetAsync(sumsq, 0, sizeof(double), s));
         return GXPO_OK;
     }
     const bool adamw = c->opt.kind == GXPO_OPT_ADAMW;
-    // AdamW sweeps that write m and v back run bulk-copy staged on long lists (default) or
-    // always (variant 3); the read-heavy deferred probe and plain GD stay register-staged.
-    if (adamw && p.write_state && ((c->variant == 0 && num_chunks >= 32LL * c->sm_count) || c->variant == 3))
-        return launch_step_bulk(c, s, descs, chunks, num_chunks, flat, p, sumsq);
+    if (step_runs_staged(c, p, num_chunks))
+        return launch_step_bulk(c, s, descs, chunks, num_chunks, flat, p, sumsq, dot_out);
     StepFn fn = pick_step(adamw, c->grad_dtype == GXPO_BF16, c->variant);
     const int ush = unit_shift_for(c, num_chunks);
     const int grid = grid_for(c, (const void*)fn, num_chunks << ush,
@@ -765,10 +776,14 @@ gxpo_status gxpo_slow_step(gxpo_ctx* c, void* stream) {
     const TensorDesc none = {};
     c->t_opt += 1;
     StepParams p = make_step_params(c, 2, 0, 0, 0, 1);
+    // diagnostics: <g0, g_slow> rides along in the staged sweep (one more read of g0);
+    // otherwise it is a pass of its own over both gradients
+    const bool want_dot = c->diag_on && !c->gslow_aliased && c->num_chunks > 0;
+    const bool dot_inside = want_dot && step_runs_staged(c, p, c->num_chunks);
     gxpo_status st = launch_step(c, (cudaStream_t)stream, c->d_descs, c->d_chunks, c->num_chunks, none, p,
-                                 c->user_sumsq ? c->user_sumsq : c->d_sumsq);
+                                 c->user_sumsq ? c->user_sumsq : c->d_sumsq, dot_inside ? c->d_diag + kDiagN : nullptr);
     if (st != GXPO_OK) { c->t_opt -= 1; return st; }
-    if (c->diag_on && !c->gslow_aliased && c->num_chunks > 0) {
+    if (want_dot && !dot_inside) {
         const bool bf16 = c->grad_dtype == GXPO_BF16;
         long long g = (long long)c->sm_count * 8;        // 64 warps per SM, one chunk each at a time
         if (g * (kThreads / 32) > c->num_chunks) g = (c->num_chunks + kThreads / 32 - 1) / (kThreads / 32);

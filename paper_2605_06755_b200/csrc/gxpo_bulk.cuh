@@ -1,6 +1,8 @@
-// Bulk-copy (TMA) staging for the fused probe + extrapolate sweep: an alternative to the
-// register-staged kernel, kept selectable (gxpo_tune variant 3) because it is the design
-// one would expect to win on this GPU and the measurement says otherwise.
+// Bulk-copy (TMA) staging for the write-heavy sweeps (the fused probe + extrapolate sweep and
+// the AdamW sweep that writes m and v back): the default for long lists, where it measures
+// 2 to 4 % faster than register staging; short lists, which cannot keep one ring per SM
+// busy, and the read-heavy deferred probe stay register-staged (gxpo_tune variant 2 forces
+// register staging, variant 3 forces this file's kernels).
 //
 // One producer thread streams whole stages (one or two 2048-element tiles of every input
 // array) into a shared-memory ring with cp.async.bulk (plain 1-D copies to this CTA only, from this GPU's own
@@ -300,23 +302,25 @@ fused_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restri
 // (three stages of 2048: 6.34; two of 8192: 6.04).  The read-heavy deferred probe (14 R +
 // 4 W) is slower staged (5.8 against 6.8 TB/s) and stays register-staged.  Consumers
 // accumulate sum(g^2) like the register-staged kernel and reduce it among themselves on a
-// named barrier (the producer warp has left by then).
+// named barrier (the producer warp has left by then).  With DOT the sweep also stages g0 and
+// accumulates <g0, g> for the diagnostics' cosine (+2 bytes per parameter for bfloat16
+// gradients instead of a separate 4-byte pass); products are summed like dot_kernel's.
 // ---------------------------------------------------------------------------
 constexpr int kStepMult = 2;       // tiles per stage
 constexpr int kStepStages = 2;
-template <bool ADAMW, typename G>
+template <bool ADAMW, typename G, bool DOT>
 struct StepLayout {
     static constexpr int kElems = kTile * kStepMult;
     static constexpr unsigned kF = kElems * sizeof(float);
     static constexpr unsigned kGb = kElems * sizeof(G);
-    static constexpr unsigned kStage = (ADAMW ? 3 : 1) * kF + kGb;
+    static constexpr unsigned kStage = (ADAMW ? 3 : 1) * kF + (DOT ? 2 : 1) * kGb;
     static constexpr unsigned kTotal = kStepStages * kStage + 2 * kMaxStages * sizeof(uint64_t) + 16;
 };
 template <typename G> struct StepUnit {
-    const float* in; float* out; float* snap; float* m; float* v; const G* g; uint16_t* wb;
+    const float* in; float* out; float* snap; float* m; float* v; const G* g; const G* g0; uint16_t* wb;
     int len, full_tiles; bool vec;
 };
-template <bool ADAMW, typename G>
+template <bool ADAMW, typename G, bool DOT>
 __device__ __forceinline__ bool step_resolve(long long c, const TensorDesc* descs, const ChunkRef* chunks,
                                              const TensorDesc& flat, const StepParams& p, int stage_elems, StepUnit<G>& U) {
     ChunkRef ref; TensorDesc d;
@@ -332,18 +336,26 @@ __device__ __forceinline__ bool step_resolve(long long c, const TensorDesc* desc
     U.m = ADAMW ? d.m + off : nullptr; U.v = ADAMW ? d.v + off : nullptr;
     const void* gsel = p.which_grad == 0 ? d.g[0] : (p.which_grad == 1 ? d.g[1] : d.g[2]);
     U.g = reinterpret_cast<const G*>(gsel) + off;
+    U.g0 = DOT ? reinterpret_cast<const G*>(d.g[0]) + off : nullptr;
     U.wb = (p.emit && d.wb) ? d.wb + off : nullptr;
     U.vec = aligned32(U.in) && aligned32(U.out) && aligned32(U.g) && (!ADAMW || (aligned32(U.m) && aligned32(U.v))) &&
-            (!p.snapshot || aligned32(U.snap)) && aligned16(U.wb);
+            (!p.snapshot || aligned32(U.snap)) && aligned16(U.wb) && (!DOT || aligned32(U.g0));
     U.full_tiles = U.vec ? U.len / stage_elems : 0;
     return true;
 }
-template <bool ADAMW, typename G>
+// <a, b> over [0, len) by the 256 consumer threads, added to acc (the short pieces that
+// bypass the ring)
+template <typename G>
+__device__ __forceinline__ void consumer_dot(const G* a, const G* b, int len, double& acc) {
+    for (int e = threadIdx.x; e < len; e += kThreads) acc += (double)ld_grad1(a + e) * (double)ld_grad1(b + e);
+}
+
+template <bool ADAMW, typename G, bool DOT>
 __global__ void __launch_bounds__(kBulkThreads, 1)
 step_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restrict__ chunks,
                  long long num_chunks, TensorDesc flat, StepParams p, double* partials, unsigned* ticket,
-                 double* sumsq_out, int* error_word) {
-    typedef StepLayout<ADAMW, G> L;
+                 double* sumsq_out, int* error_word, double* dot_partials, double* dot_out) {
+    typedef StepLayout<ADAMW, G, DOT> L;
     constexpr int kStages = kStepStages;
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ double red[8];
@@ -363,7 +375,7 @@ step_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restric
         unsigned it = 0; bool ok = true;
         for (long long c = blockIdx.x; c < num_chunks && ok; c += gridDim.x) {
             StepUnit<G> U;
-            if (!step_resolve<ADAMW, G>(c, descs, chunks, flat, p, L::kElems, U)) continue;
+            if (!step_resolve<ADAMW, G, DOT>(c, descs, chunks, flat, p, L::kElems, U)) continue;
             for (int j = 0; j < U.full_tiles; ++j, ++it) {
                 const unsigned s = it % kStages, n = it / kStages;
                 if (n > 0 && !mbar_wait_bounded(empty + s, (n - 1) & 1, stop, kWaitLimit)) { ok = false; break; }
@@ -373,7 +385,8 @@ step_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restric
                 unsigned o = 0;
                 bulk_load(st, U.in + e, L::kF, full + s); o += L::kF;
                 if (ADAMW) { bulk_load(st + o, U.m + e, L::kF, full + s); o += L::kF; bulk_load(st + o, U.v + e, L::kF, full + s); o += L::kF; }
-                bulk_load(st + o, U.g + e, L::kGb, full + s);
+                bulk_load(st + o, U.g + e, L::kGb, full + s); o += L::kGb;
+                if (DOT) bulk_load(st + o, U.g0 + e, L::kGb, full + s);
             }
         }
         if (!ok) {
@@ -386,11 +399,15 @@ step_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restric
         return;
     }
     const float gscale = p.gscale ? __ldg(p.gscale) : 1.0f;
-    double acc = 0.0; unsigned it = 0; bool alive = true;
+    double acc = 0.0, accd = 0.0; unsigned it = 0; bool alive = true;
     for (long long c = blockIdx.x; c < num_chunks && alive; c += gridDim.x) {
         StepUnit<G> U;
-        if (!step_resolve<ADAMW, G>(c, descs, chunks, flat, p, L::kElems, U)) continue;
-        if (!U.vec) { step_chunk_scalar<ADAMW, G>(U.out, U.in, U.snap, U.m, U.v, U.g, U.len, p, gscale, acc, U.wb); continue; }
+        if (!step_resolve<ADAMW, G, DOT>(c, descs, chunks, flat, p, L::kElems, U)) continue;
+        if (!U.vec) {
+            step_chunk_scalar<ADAMW, G>(U.out, U.in, U.snap, U.m, U.v, U.g, U.len, p, gscale, acc, U.wb);
+            if (DOT) consumer_dot(U.g0, U.g, U.len, accd);
+            continue;
+        }
         for (int j = 0; j < U.full_tiles; ++j, ++it) {
             const unsigned s = it % kStages, n = it / kStages;
             if (!mbar_wait_bounded(full + s, n & 1, stop, kWaitLimit)) { *stop = 1; atomicExch(error_word, 1); alive = false; break; }
@@ -402,7 +419,14 @@ step_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restric
                 FVec<8> th, mm, vv;
                 th = lds_f8(reinterpret_cast<const float*>(st) + tt); o += L::kF;
                 if (ADAMW) { mm = lds_f8(reinterpret_cast<const float*>(st + o) + tt); o += L::kF; vv = lds_f8(reinterpret_cast<const float*>(st + o) + tt); o += L::kF; }
-                const FVec<8> gg = lds_g8(reinterpret_cast<const G*>(st + o) + tt);
+                const FVec<8> gg = lds_g8(reinterpret_cast<const G*>(st + o) + tt); o += L::kGb;
+                if (DOT) {
+                    const FVec<8> g0 = lds_g8(reinterpret_cast<const G*>(st + o) + tt);
+                    float dq = 0.0f;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) dq = fmaf(g0.x[i], gg.x[i], dq);
+                    accd += (double)dq;
+                }
                 const int e = j * L::kElems + tt;
                 if (U.snap) st_f(U.snap + e, th);
                 float sq = 0.0f;
@@ -418,20 +442,37 @@ step_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restric
         }
         if (!alive) break;
         const int done = U.full_tiles * L::kElems;
-        if (done < U.len)
+        if (done < U.len) {
             step_chunk_vec<ADAMW, G, 8>(U.out + done, U.in + done, U.snap ? U.snap + done : nullptr, ADAMW ? U.m + done : nullptr,
                                         ADAMW ? U.v + done : nullptr, U.g + done, U.len - done, p, gscale, acc, U.wb ? U.wb + done : nullptr);
+            if (DOT) consumer_dot(U.g0 + done, U.g + done, U.len - done, accd);
+        }
     }
-    if (p.want_norm) {
+    if (p.want_norm) {                                   // DOT comes only with want_norm
         const double tot = consumer_sum(acc, red);
-        if (threadIdx.x == 0) { partials[blockIdx.x] = tot; __threadfence(); is_last = (atomicAdd(ticket, 1u) == gridDim.x - 1); }
+        double totd = 0.0;
+        if (DOT) totd = consumer_sum(accd, red);
+        if (threadIdx.x == 0) {
+            partials[blockIdx.x] = tot;
+            if (DOT) dot_partials[blockIdx.x] = totd;
+            __threadfence();
+            is_last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+        }
         asm volatile("bar.sync 1, %0;" :: "r"(kThreads) : "memory");
         if (is_last) {
             __threadfence();
-            double sum = 0.0;
-            for (unsigned i = threadIdx.x; i < gridDim.x; i += kThreads) sum += __ldcg(partials + i);
+            double sum = 0.0, sumd = 0.0;
+            for (unsigned i = threadIdx.x; i < gridDim.x; i += kThreads) {
+                sum += __ldcg(partials + i);
+                if (DOT) sumd += __ldcg(dot_partials + i);
+            }
             sum = consumer_sum(sum, red);
-            if (threadIdx.x == 0) { *sumsq_out = sum; *ticket = 0u; }
+            if (DOT) sumd = consumer_sum(sumd, red);
+            if (threadIdx.x == 0) {
+                *sumsq_out = sum;
+                if (DOT) *dot_out = sumd;
+                *ticket = 0u;
+            }
         }
     }
 }
