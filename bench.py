@@ -66,6 +66,8 @@ def parse_args():
     ap.add_argument("--emit-bf16", action="store_true",
                     help="also keep bfloat16 model-weight copies (gxpo_bind_model_weights, bf16-only theta1): "
                          "16 + 30 + 28 = 74 B/param, and the caller needs no cast sweeps")
+    ap.add_argument("--no-persist", action="store_true",
+                    help="do not promise that g0 and g1 outlive the slow step (72 instead of 68 B/param in the deferred flow)")
     ap.add_argument("--diagnostics", action="store_true",
                     help="gather the per-step diagnostics too (adds a 4 B/param <g0, g_slow> pass after the slow step)")
     ap.add_argument("--no-e2e", action="store_true")
@@ -312,6 +314,9 @@ def run_ours(args):
     ctx.bind(ptrs)
     diag = bool(getattr(args, "diagnostics", False)) and not args.fallback
     ctx.enable_diagnostics(diag)
+    # the benchmark's g0 and g1 are buffers of their own that nothing overwrites: say so
+    persist = not getattr(args, "no_persist", False) and args.flow == "deferred" and not alias and not args.fallback
+    ctx.set_gradients_persist(persist)
     if emit:
         weights = torch.empty(d, dtype=torch.bfloat16, device="cuda")
         offs, acc = [], 0
@@ -323,7 +328,11 @@ def run_ours(args):
         ctx.set_sumsq_buffer(sumsq.data_ptr())
 
     flow = args.flow
-    names = {"deferred": ["probe_step0_deferred", "probe_extrapolate_deferred", "slow_step"],
+    n_chunks = sum((k + 32767) // 32768 for _, k in shapes)
+    staged = args.variant == 3 or (args.variant == 0 and n_chunks >= 32 * props.multi_processor_count)
+    lag = persist and staged and not diag     # the fused sweep leaves m, v unwritten; the slow sweep replays from g0, g1
+    names = {"deferred": (["probe_step0_deferred", "probe_extrapolate_nostate", "slow_step_replay"] if lag else
+                          ["probe_step0_deferred", "probe_extrapolate_deferred", "slow_step"]),
              "fused": ["probe_step0", "probe_extrapolate", "slow_step"],
              "unfused": ["probe_step0", "probe_step1", "extrapolate", "slow_step"]}[flow]
     if args.fallback:
@@ -404,13 +413,16 @@ def run_ours(args):
         alg_bytes["probe_extrapolate_deferred"] += 2
         alg_bytes["slow_step"] += 2
     kernel_of = dict(KERNEL_OF)
-    n_chunks = sum((k + 32767) // 32768 for _, k in shapes)
-    staged = args.variant == 3 or (args.variant == 0 and n_chunks >= 32 * props.multi_processor_count)
+    alg_bytes["probe_extrapolate_nostate"] = alg_bytes["probe_extrapolate_deferred"] - 8   # m, v not written
+    alg_bytes["slow_step_replay"] = alg_bytes["slow_step"] + 4              # g0 and g1 read once more
     if diag and not alias:      # <g0, g_slow>, timed with the slow step: g0 read once more inside the staged
-        alg_bytes["slow_step"] += 2 if staged else 4      # sweep, else a pass of its own over both gradients
+        alg_bytes["slow_step"] += 2 if staged else 4      # sweep (already there when it replays), else a pass
+                                                          # of its own over both gradients
     if staged:
         # the fused sweep runs in its bulk-copy staged kernel (the library's default for long lists)
         kernel_of["probe_extrapolate"] = kernel_of["probe_extrapolate_deferred"] = "fused_bulk_kernel"
+        kernel_of["probe_extrapolate_nostate"] = "fused_bulk_light_kernel"
+        kernel_of["slow_step_replay"] = "step_bulk_kernel"
         for nm in ("probe_step0", "probe_step1", "slow_step", "fallback_step"):   # AdamW sweeps that write m, v back
             kernel_of[nm] = "step_bulk_kernel"
     kernels = {nm: {"kernel": kernel_of[nm], "ms": ms, "bytes_per_param": alg_bytes[nm],
@@ -443,10 +455,12 @@ def run_ours(args):
                    "K": args.K, "alpha": args.alpha, "lr": args.lr, "grad_dtype": "bf16",
                    "placement": ["pingpong", "snapshot"][args.placement],
                    "step": "fallback (single pass)" if args.fallback else
-                   {"deferred": "active (probe with deferred state, probe+extrapolate in one sweep, slow step, gate)",
+                   {"deferred": ("active (probe with deferred state, probe+extrapolate in one sweep with m, v still unwritten, "
+                                 "slow step replaying both moment updates, gate)") if lag else
+                                "active (probe with deferred state, probe+extrapolate in one sweep, slow step, gate)",
                     "fused": "active (probe, probe+extrapolate in one sweep, slow step, gate)",
                     "unfused": "active (probe, probe, extrapolate, slow step, gate)"}[flow],
-                   "bf16_model_weight_copies": emit, "diagnostics": diag, "g_slow_aliases_g0": alias, "l2": "inputs larger than L2 (no flush needed)",
+                   "bf16_model_weight_copies": emit, "diagnostics": diag, "gradients_persist": persist, "g_slow_aliases_g0": alias, "l2": "inputs larger than L2 (no flush needed)",
                    "parallelism": f"dp{world} (independent shards, one 8-byte all-reduce per step)" if world > 1 else "1 GPU"},
         "hbm_gbs_whole_step": whole_gbs, "hbm_frac_whole_step": whole_gbs / peak,
         "hbm_frac_of_8tbs_nominal": whole_gbs / 8000.0,

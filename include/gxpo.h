@@ -198,6 +198,21 @@ gxpo_status gxpo_probe_extrapolate(gxpo_ctx* ctx, void* stream);
  * state: IDLE -> PROBED0_DEFERRED; from there only gxpo_probe_extrapolate is legal. */
 gxpo_status gxpo_probe_step_deferred(gxpo_ctx* ctx, void* stream);
 
+/* A promise about the caller's gradient buffers, off by default: on != 0 says that g0 and
+ * g1 still hold this step's gradients while gxpo_slow_step's sweep runs (nothing reuses
+ * them between the backward passes, and g_slow has a buffer of its own).  After
+ * gxpo_probe_step_deferred, gxpo_probe_extrapolate may then leave m and v unwritten once
+ * more, and the slow step's sweep replays both probe steps' moment updates in registers from
+ * g0 and g1 before it takes its own step: 18 + 20 + 30 = 68 instead of 72 bytes per
+ * parameter, bit-identical theta, m and v.  The library uses this where it pays (AdamW on
+ * lists long enough for the shared-memory staged sweep, see gxpo_tune, with diagnostics
+ * off) and never when some tensor's g_slow pointer equals its g0 or g1 pointer; elsewhere
+ * the promise changes nothing.  Between gxpo_probe_extrapolate and gxpo_slow_step m and v in memory are then
+ * two steps behind; a caller who breaks the promise gets wrong moments, not an error.
+ * Paper: no counterpart (Algorithm 1 does not say where the optimizer state lives between
+ * its three steps).  Errors: STATE mid-step. */
+gxpo_status gxpo_set_gradients_persist(gxpo_ctx* ctx, int on);
+
 /* Algorithm 1, "slow correction": theta^{t+1} <- OptimStep(theta-tilde, g_slow), in
  * place in `theta`, and sum(g_slow^2) accumulated in the same sweep (float64,
  * deterministic for a fixed launch shape).  state: EXTRAPOLATED -> SLOW_DONE. */

@@ -81,6 +81,7 @@ _sigs = {
     "gxpo_set_grad_scale": (ctypes.c_int, [_vp, ctypes.c_int, _vp]),
     "gxpo_clip_grad_norm": (ctypes.c_int, [_vp, ctypes.c_int, ctypes.c_double, _vp]),
     "gxpo_enable_diagnostics": (ctypes.c_int, [_vp, ctypes.c_int]),
+    "gxpo_set_gradients_persist": (ctypes.c_int, [_vp, ctypes.c_int]),
     "gxpo_get_diagnostics": (ctypes.c_int, [_vp, _vp, ctypes.POINTER(Diagnostics)]),
     "gxpo_gate_peek": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_int),
                                       ctypes.POINTER(ctypes.c_longlong),
@@ -254,6 +255,9 @@ class Context:
 
     def enable_diagnostics(self, on: bool = True):
         self._check(_lib.gxpo_enable_diagnostics(self._h, 1 if on else 0))
+
+    def set_gradients_persist(self, on: bool):
+        self._check(_lib.gxpo_set_gradients_persist(self._h, 1 if on else 0))
 
     def get_diagnostics(self, stream=None) -> Diagnostics:
         out = Diagnostics()

@@ -82,6 +82,9 @@ struct gxpo_ctx {
     int diag_on;
     int diag_ready;                    // 1 once an active step with diagnostics has completed
     int gslow_aliased;                 // some tensor's g_slow shares g0's buffer: no <g0, g_slow>
+    int gslow_shares_probe;            // some tensor's g_slow shares g0's or g1's buffer
+    int grads_persist;                 // the caller promised that g0 and g1 outlive the slow step's sweep
+    int state_lag;                     // this step's fused sweep left m and v unwritten: the slow step replays
     double* d_diag;                    // kDiagN sums + <g0, g_slow>
     double* d_diag_partials;           // kDiagN x kMaxGrid
     DiagResult* d_diag_result;
@@ -248,8 +251,15 @@ template <typename G>
 gxpo_status launch_step_bulk_t(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
                                long long num_chunks, const TensorDesc& flat, const StepParams& p, double* sumsq,
                                double* dot_out) {
-    StepBulkFn fn = dot_out ? step_bulk_kernel<true, G, true> : step_bulk_kernel<true, G, false>;
-    const int smem = dot_out ? (int)StepLayout<true, G, true>::kTotal : (int)StepLayout<true, G, false>::kTotal;
+    StepBulkFn fn;
+    int smem;
+#define GXPO_STEP_MODE(M) { fn = step_bulk_kernel<true, G, M>; smem = (int)StepLayout<true, G, M>::kTotal; }
+    switch ((dot_out ? kStepDot : 0) | (p.replay ? kStepReplay : 0)) {
+        case 0: GXPO_STEP_MODE(0) break;
+        case kStepDot: GXPO_STEP_MODE(kStepDot) break;
+        default: GXPO_STEP_MODE(kStepReplay) break;       // replay never comes with diagnostics
+    }
+#undef GXPO_STEP_MODE
     int resident = 0;
     for (int i = 0; i < c->occ_n; ++i)
         if (c->occ_key[i] == (const void*)fn) resident = c->occ_val[i];
@@ -296,7 +306,7 @@ gxpo_status launch_step(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, co
         return GXPO_OK;
     }
     const bool adamw = c->opt.kind == GXPO_OPT_ADAMW;
-    if (step_runs_staged(c, p, num_chunks))
+    if (p.replay || step_runs_staged(c, p, num_chunks))      // only the staged kernel can replay
         return launch_step_bulk(c, s, descs, chunks, num_chunks, flat, p, sumsq, dot_out);
     StepFn fn = pick_step(adamw, c->grad_dtype == GXPO_BF16, c->variant);
     const int ush = unit_shift_for(c, num_chunks);
@@ -330,7 +340,15 @@ template <bool ADAMW, typename G, bool DEFER>
 gxpo_status launch_bulk_t(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
                           long long num_chunks, const TensorDesc& flat, const FusedParams& p, bool diag) {
     BulkFn fn = diag ? fused_bulk_kernel<ADAMW, G, DEFER, true> : fused_bulk_kernel<ADAMW, G, DEFER, false>;
-    const int smem = (int)BulkLayout<ADAMW, G, DEFER>::kTotal;
+    int smem = (int)BulkLayout<ADAMW, G, DEFER>::kTotal;
+    int want_per_sm = kDefaultCtasBulk;
+    if constexpr (ADAMW && DEFER) {
+        if (!p.step.write_state && !diag) {   // m and v stay unwritten: the latency-bound shape, two CTAs per SM
+            fn = fused_bulk_light_kernel<G>;                      // (with diagnostics it would not fit the registers)
+            smem = (int)BulkLayout<true, G, true, true>::kTotal;
+            want_per_sm = 2;
+        }
+    }
     // first launch of this instantiation in this context: allow the ring's shared memory and
     // find out how many CTAs fit; remembered in the occupancy cache afterwards
     int resident = 0;
@@ -342,7 +360,7 @@ gxpo_status launch_bulk_t(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, 
             resident = 1;
         if (c->occ_n < 32) { c->occ_key[c->occ_n] = (const void*)fn; c->occ_val[c->occ_n] = resident; c->occ_n += 1; }
     }
-    int per_sm = c->ctas_per_sm > 0 ? c->ctas_per_sm : kDefaultCtasBulk;
+    int per_sm = c->ctas_per_sm > 0 ? c->ctas_per_sm : want_per_sm;
     if (per_sm > resident) per_sm = resident;
     long long g = (long long)c->sm_count * per_sm;
     if (g > num_chunks) g = num_chunks;
@@ -616,7 +634,7 @@ gxpo_status gxpo_bind(gxpo_ctx* c, const gxpo_tensor* list, int count) {
     std::vector<TensorDesc> descs((size_t)count);
     std::vector<ChunkRef> chunks;
     long long total = 0;
-    int aliased = 0;
+    int aliased = 0, shares_probe = 0;
     for (int i = 0; i < count; ++i) {
         gxpo_status s = check_tensor(c, list[i], i, true);
         if (s != GXPO_OK) return s;
@@ -626,6 +644,7 @@ gxpo_status gxpo_bind(gxpo_ctx* c, const gxpo_tensor* list, int count) {
         d.n = list[i].n;
         total += d.n;
         if (d.n > 0 && d.g[2] == d.g[0]) aliased = 1;
+        if (d.n > 0 && (d.g[2] == d.g[0] || d.g[2] == d.g[1])) shares_probe = 1;
     }
     chunks.reserve((size_t)(total / kChunk + count));
     for (int i = 0; i < count; ++i) {
@@ -648,6 +667,8 @@ gxpo_status gxpo_bind(gxpo_ctx* c, const gxpo_tensor* list, int count) {
     c->num_tensors = count;
     c->total_params = total;
     c->gslow_aliased = aliased;
+    c->gslow_shares_probe = shares_probe;
+    c->state_lag = 0;
     c->diag_ready = 0;
     c->only_bf16_theta1 = 0;
     if (!c->h_descs) c->h_descs = new (std::nothrow) std::vector<TensorDesc>();
@@ -763,9 +784,20 @@ gxpo_status gxpo_probe_extrapolate(gxpo_ctx* c, void* stream) {
     c->t_opt += 1;
     p.step = (place == GXPO_PLACE_PINGPONG) ? make_step_params(c, 1, 1, 1, 0, 0) : make_step_params(c, 1, 0, 0, 0, 0);
     p.ex = make_extrap_params(c, place);
+    // With the caller's promise that g0 and g1 outlive the slow step's sweep, m and v can stay
+    // unwritten once more: the slow step's staged sweep replays both moment updates from g0
+    // and g1 (8 bytes of writes saved here, 4 bytes of reads added there).  Only where that
+    // sweep will run staged, never when g_slow lands in g0's or g1's buffer, and not with
+    // diagnostics on (their arithmetic, not the state writes, then bounds this sweep).
+    StepParams slow = p.step;
+    slow.write_state = 1;
+    const bool lag = defer && c->grads_persist && !c->gslow_shares_probe && c->opt.kind == GXPO_OPT_ADAMW &&
+                     !c->diag_on && step_runs_staged(c, slow, c->num_chunks);
+    if (lag) p.step.write_state = 0;
     gxpo_status st = launch_fused(c, (cudaStream_t)stream, c->d_descs, c->d_chunks, c->num_chunks, none, p, defer,
                                   c->diag_on != 0);
     if (st != GXPO_OK) { c->t_opt -= 1; return st; }
+    c->state_lag = lag ? 1 : 0;
     c->phase = EXTRAPOLATED;
     return GXPO_OK;
 }
@@ -778,11 +810,17 @@ gxpo_status gxpo_slow_step(gxpo_ctx* c, void* stream) {
     StepParams p = make_step_params(c, 2, 0, 0, 0, 1);
     // diagnostics: <g0, g_slow> rides along in the staged sweep (one more read of g0);
     // otherwise it is a pass of its own over both gradients
+    if (c->state_lag) {
+        p.replay = 1;
+        p.gscale_r0 = c->gscale[0];
+        p.gscale_r1 = c->gscale[1];
+    }
     const bool want_dot = c->diag_on && !c->gslow_aliased && c->num_chunks > 0;
-    const bool dot_inside = want_dot && step_runs_staged(c, p, c->num_chunks);
+    const bool dot_inside = want_dot && !p.replay && step_runs_staged(c, p, c->num_chunks);
     gxpo_status st = launch_step(c, (cudaStream_t)stream, c->d_descs, c->d_chunks, c->num_chunks, none, p,
                                  c->user_sumsq ? c->user_sumsq : c->d_sumsq, dot_inside ? c->d_diag + kDiagN : nullptr);
     if (st != GXPO_OK) { c->t_opt -= 1; return st; }
+    c->state_lag = 0;
     if (want_dot && !dot_inside) {
         const bool bf16 = c->grad_dtype == GXPO_BF16;
         long long g = (long long)c->sm_count * 8;        // 64 warps per SM, one chunk each at a time
@@ -877,6 +915,13 @@ gxpo_status gxpo_enable_diagnostics(gxpo_ctx* c, int on) {
     if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "diagnostics can only be switched between steps");
     c->diag_on = on ? 1 : 0;
     c->diag_ready = 0;
+    return GXPO_OK;
+}
+
+gxpo_status gxpo_set_gradients_persist(gxpo_ctx* c, int on) {
+    if (!c) return GXPO_ERR_INVALID_ARG;
+    if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "the promise can only be changed between steps");
+    c->grads_persist = on ? 1 : 0;
     return GXPO_OK;
 }
 

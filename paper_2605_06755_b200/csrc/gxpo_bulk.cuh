@@ -127,9 +127,11 @@ __device__ __forceinline__ double consumer_sum(double x, double* smem8) {
 // in as few, as large pieces as possible.  Deferred sweep (5 arrays): 2 stages of 4096
 // elements 6.62 TB/s, 3 of 2048 6.53, 2 of 2048 5.77, 4 of 2048 6.10, 3 of 4096 6.09.  The
 // non-deferred sweep (6 arrays) does best with 3 stages of 2048.
-template <bool ADAMW, typename G, bool DEFER>
+// LIGHT (deferred AdamW sweep that leaves m and v unwritten: 16 R + 4 W) is bound by
+// latency rather than by the write path: two CTAs per SM, each with 2 stages of 2048.
+template <bool ADAMW, typename G, bool DEFER, bool LIGHT = false>
 struct BulkLayout {
-    static constexpr int kMult = DEFER ? 2 : 1;                  // tiles per stage
+    static constexpr int kMult = (DEFER && !LIGHT) ? 2 : 1;      // tiles per stage
     static constexpr int kStagesN = DEFER ? 2 : 3;
     static constexpr int kElems = kTile * kMult;
     static constexpr unsigned kF = kElems * sizeof(float);
@@ -138,12 +140,12 @@ struct BulkLayout {
     static constexpr unsigned kTotal = kStagesN * kStage + 2 * kMaxStages * sizeof(uint64_t) + 16;
 };
 
-template <bool ADAMW, typename G, bool DEFER, bool DIAG>
-__global__ void __launch_bounds__(kBulkThreads, 1)
-fused_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restrict__ chunks,
-                  long long num_chunks, TensorDesc flat, FusedParams p, int* error_word,
-                  double* diag_partials, unsigned* ticket, double* diag_out) {
-    typedef BulkLayout<ADAMW, G, DEFER> L;
+template <bool ADAMW, typename G, bool DEFER, bool DIAG, bool LIGHT>
+__device__ __forceinline__ void fused_bulk_body(const TensorDesc* __restrict__ descs, const ChunkRef* __restrict__ chunks,
+                                                long long num_chunks, const TensorDesc& flat, const FusedParams& p,
+                                                int* error_word, double* diag_partials, unsigned* ticket,
+                                                double* diag_out) {
+    typedef BulkLayout<ADAMW, G, DEFER, LIGHT> L;
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int kStages = L::kStagesN;
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStages * L::kStage);
@@ -218,7 +220,7 @@ fused_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restri
                                                                 __fmul_rn(ld_grad1(U.g1 + e), gs1), p, &acc);
                 U.out[e] = x;
                 if (U.wb) U.wb[e] = to_bf16(x);
-                if (ADAMW) { U.m[e] = mm; U.v[e] = vv; }
+                if (ADAMW && !LIGHT && p.step.write_state) { U.m[e] = mm; U.v[e] = vv; }
             }
             continue;
         }
@@ -253,7 +255,7 @@ fused_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restri
             extrapolate_vec<8, DIAG>(a1, a0, b0, b1, p.ex, &acc);
             st_f(U.out + e, a1);
             if (U.wb) st_bf16(U.wb + e, a1);
-            if (ADAMW) { st_f(U.m + e, mm); st_f(U.v + e, vv); }
+            if (ADAMW && !LIGHT && p.step.write_state) { st_f(U.m + e, mm); st_f(U.v + e, vv); }
             }
             // Hand the stage back only now: every lane's stores depend on what it read from
             // the stage, so by this point the shared-memory reads have certainly completed.
@@ -295,6 +297,25 @@ fused_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restri
     }
 }
 
+template <bool ADAMW, typename G, bool DEFER, bool DIAG>
+__global__ void __launch_bounds__(kBulkThreads, 1)
+fused_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restrict__ chunks,
+                  long long num_chunks, TensorDesc flat, FusedParams p, int* error_word,
+                  double* diag_partials, unsigned* ticket, double* diag_out) {
+    fused_bulk_body<ADAMW, G, DEFER, DIAG, false>(descs, chunks, num_chunks, flat, p, error_word, diag_partials, ticket, diag_out);
+}
+
+// The LIGHT shape, two CTAs per SM: 18 warps put 5 on one scheduler, whose 16384 registers
+// then allow 96 per thread (the compiler spills 76 bytes; measured 23.7 ms against 24.6 with
+// one CTA and against 29.2 ms at 112 registers, where only one CTA fits).
+template <typename G>
+__global__ void __launch_bounds__(kBulkThreads, 2)
+fused_bulk_light_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restrict__ chunks,
+                        long long num_chunks, TensorDesc flat, FusedParams p, int* error_word,
+                        double* diag_partials, unsigned* ticket, double* diag_out) {
+    fused_bulk_body<true, G, true, false, true>(descs, chunks, num_chunks, flat, p, error_word, diag_partials, ticket, diag_out);
+}
+
 // ---------------------------------------------------------------------------
 // The AdamW sweep with the same staging, for the calls that write m and v back (slow
 // step, fallback step, non-deferred probe steps): 14 R + 12 W per parameter.  Measured on a
@@ -302,25 +323,32 @@ fused_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restri
 // (three stages of 2048: 6.34; two of 8192: 6.04).  The read-heavy deferred probe (14 R +
 // 4 W) is slower staged (5.8 against 6.8 TB/s) and stays register-staged.  Consumers
 // accumulate sum(g^2) like the register-staged kernel and reduce it among themselves on a
-// named barrier (the producer warp has left by then).  With DOT the sweep also stages g0 and
-// accumulates <g0, g> for the diagnostics' cosine (+2 bytes per parameter for bfloat16
-// gradients instead of a separate 4-byte pass); products are summed like dot_kernel's.
+// named barrier (the producer warp has left by then).
+// MODE bit kStepDot: the sweep also stages g0 and accumulates <g0, g> for the diagnostics'
+// cosine (+2 bytes per parameter for bfloat16 gradients instead of a separate 4-byte pass);
+// products are summed like dot_kernel's.
+// MODE bit kStepReplay: m and v are still those from before the two probe steps (the fused
+// sweep left them unwritten as well); g0 and g1 are staged too and both moment updates are
+// replayed in registers before the step itself: 18 R + 12 W, and the fused sweep before it
+// saves its 8 bytes of state writes.
 // ---------------------------------------------------------------------------
+constexpr int kStepDot = 1, kStepReplay = 2;
 constexpr int kStepMult = 2;       // tiles per stage
 constexpr int kStepStages = 2;
-template <bool ADAMW, typename G, bool DOT>
+template <bool ADAMW, typename G, int MODE>
 struct StepLayout {
     static constexpr int kElems = kTile * kStepMult;
     static constexpr unsigned kF = kElems * sizeof(float);
     static constexpr unsigned kGb = kElems * sizeof(G);
-    static constexpr unsigned kStage = (ADAMW ? 3 : 1) * kF + (DOT ? 2 : 1) * kGb;
+    static constexpr int kGrads = 1 + (MODE != 0 ? 1 : 0) + ((MODE & kStepReplay) ? 1 : 0);   // g [g0 [g1]]
+    static constexpr unsigned kStage = (ADAMW ? 3 : 1) * kF + kGrads * kGb;
     static constexpr unsigned kTotal = kStepStages * kStage + 2 * kMaxStages * sizeof(uint64_t) + 16;
 };
 template <typename G> struct StepUnit {
-    const float* in; float* out; float* snap; float* m; float* v; const G* g; const G* g0; uint16_t* wb;
+    const float* in; float* out; float* snap; float* m; float* v; const G* g; const G* g0; const G* g1; uint16_t* wb;
     int len, full_tiles; bool vec;
 };
-template <bool ADAMW, typename G, bool DOT>
+template <bool ADAMW, typename G, int MODE>
 __device__ __forceinline__ bool step_resolve(long long c, const TensorDesc* descs, const ChunkRef* chunks,
                                              const TensorDesc& flat, const StepParams& p, int stage_elems, StepUnit<G>& U) {
     ChunkRef ref; TensorDesc d;
@@ -336,10 +364,11 @@ __device__ __forceinline__ bool step_resolve(long long c, const TensorDesc* desc
     U.m = ADAMW ? d.m + off : nullptr; U.v = ADAMW ? d.v + off : nullptr;
     const void* gsel = p.which_grad == 0 ? d.g[0] : (p.which_grad == 1 ? d.g[1] : d.g[2]);
     U.g = reinterpret_cast<const G*>(gsel) + off;
-    U.g0 = DOT ? reinterpret_cast<const G*>(d.g[0]) + off : nullptr;
+    U.g0 = MODE ? reinterpret_cast<const G*>(d.g[0]) + off : nullptr;
+    U.g1 = (MODE & kStepReplay) ? reinterpret_cast<const G*>(d.g[1]) + off : nullptr;
     U.wb = (p.emit && d.wb) ? d.wb + off : nullptr;
     U.vec = aligned32(U.in) && aligned32(U.out) && aligned32(U.g) && (!ADAMW || (aligned32(U.m) && aligned32(U.v))) &&
-            (!p.snapshot || aligned32(U.snap)) && aligned16(U.wb) && (!DOT || aligned32(U.g0));
+            (!p.snapshot || aligned32(U.snap)) && aligned16(U.wb) && aligned32(U.g0) && aligned32(U.g1);   // null passes
     U.full_tiles = U.vec ? U.len / stage_elems : 0;
     return true;
 }
@@ -350,12 +379,38 @@ __device__ __forceinline__ void consumer_dot(const G* a, const G* b, int len, do
     for (int e = threadIdx.x; e < len; e += kThreads) acc += (double)ld_grad1(a + e) * (double)ld_grad1(b + e);
 }
 
-template <bool ADAMW, typename G, bool DOT>
+// The pieces that bypass the ring, replay mode: advance m and v in place with g0 and g1, after
+// which the ordinary code paths apply.  Every thread advances exactly the elements it will
+// read back itself (VEC: the vectors and the tail element step_chunk_vec<.., 8> gives it;
+// otherwise step_chunk_scalar's stride), so no barrier is needed, only program order.
+template <typename G, bool VEC>
+__device__ __forceinline__ void consumer_replay(float* m, float* v, const G* g0, const G* g1, int len,
+                                                const StepParams& p, float gs0, float gs1) {
+    auto one = [&](int e) {
+        float mm = m[e], vv = v[e];
+        advance_moments_elem(mm, vv, __fmul_rn(ld_grad1(g0 + e), gs0), p);
+        advance_moments_elem(mm, vv, __fmul_rn(ld_grad1(g1 + e), gs1), p);
+        m[e] = mm; v[e] = vv;
+    };
+    if (VEC) {
+        const int nvec = len / 8;
+        for (int iv = threadIdx.x; iv < nvec; iv += kThreads)
+            for (int i = 0; i < 8; ++i) one(iv * 8 + i);
+        const int e = nvec * 8 + threadIdx.x;
+        if (e < len) one(e);
+    } else {
+        for (int e = threadIdx.x; e < len; e += kThreads) one(e);
+    }
+    asm volatile("" ::: "memory");          // the loads that follow are asm statements
+}
+
+template <bool ADAMW, typename G, int MODE>
 __global__ void __launch_bounds__(kBulkThreads, 1)
 step_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restrict__ chunks,
                  long long num_chunks, TensorDesc flat, StepParams p, double* partials, unsigned* ticket,
                  double* sumsq_out, int* error_word, double* dot_partials, double* dot_out) {
-    typedef StepLayout<ADAMW, G, DOT> L;
+    typedef StepLayout<ADAMW, G, MODE> L;
+    constexpr bool DOT = (MODE & kStepDot) != 0, REPLAY = (MODE & kStepReplay) != 0;
     constexpr int kStages = kStepStages;
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ double red[8];
@@ -375,7 +430,7 @@ step_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restric
         unsigned it = 0; bool ok = true;
         for (long long c = blockIdx.x; c < num_chunks && ok; c += gridDim.x) {
             StepUnit<G> U;
-            if (!step_resolve<ADAMW, G, DOT>(c, descs, chunks, flat, p, L::kElems, U)) continue;
+            if (!step_resolve<ADAMW, G, MODE>(c, descs, chunks, flat, p, L::kElems, U)) continue;
             for (int j = 0; j < U.full_tiles; ++j, ++it) {
                 const unsigned s = it % kStages, n = it / kStages;
                 if (n > 0 && !mbar_wait_bounded(empty + s, (n - 1) & 1, stop, kWaitLimit)) { ok = false; break; }
@@ -386,7 +441,8 @@ step_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restric
                 bulk_load(st, U.in + e, L::kF, full + s); o += L::kF;
                 if (ADAMW) { bulk_load(st + o, U.m + e, L::kF, full + s); o += L::kF; bulk_load(st + o, U.v + e, L::kF, full + s); o += L::kF; }
                 bulk_load(st + o, U.g + e, L::kGb, full + s); o += L::kGb;
-                if (DOT) bulk_load(st + o, U.g0 + e, L::kGb, full + s);
+                if (MODE) { bulk_load(st + o, U.g0 + e, L::kGb, full + s); o += L::kGb; }
+                if (REPLAY) bulk_load(st + o, U.g1 + e, L::kGb, full + s);
             }
         }
         if (!ok) {
@@ -399,11 +455,14 @@ step_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restric
         return;
     }
     const float gscale = p.gscale ? __ldg(p.gscale) : 1.0f;
+    const float gs0 = (REPLAY && p.gscale_r0) ? __ldg(p.gscale_r0) : 1.0f;
+    const float gs1 = (REPLAY && p.gscale_r1) ? __ldg(p.gscale_r1) : 1.0f;
     double acc = 0.0, accd = 0.0; unsigned it = 0; bool alive = true;
     for (long long c = blockIdx.x; c < num_chunks && alive; c += gridDim.x) {
         StepUnit<G> U;
-        if (!step_resolve<ADAMW, G, DOT>(c, descs, chunks, flat, p, L::kElems, U)) continue;
+        if (!step_resolve<ADAMW, G, MODE>(c, descs, chunks, flat, p, L::kElems, U)) continue;
         if (!U.vec) {
+            if (REPLAY) consumer_replay<G, false>(U.m, U.v, U.g0, U.g1, U.len, p, gs0, gs1);
             step_chunk_scalar<ADAMW, G>(U.out, U.in, U.snap, U.m, U.v, U.g, U.len, p, gscale, acc, U.wb);
             if (DOT) consumer_dot(U.g0, U.g, U.len, accd);
             continue;
@@ -420,12 +479,22 @@ step_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restric
                 th = lds_f8(reinterpret_cast<const float*>(st) + tt); o += L::kF;
                 if (ADAMW) { mm = lds_f8(reinterpret_cast<const float*>(st + o) + tt); o += L::kF; vv = lds_f8(reinterpret_cast<const float*>(st + o) + tt); o += L::kF; }
                 const FVec<8> gg = lds_g8(reinterpret_cast<const G*>(st + o) + tt); o += L::kGb;
-                if (DOT) {
-                    const FVec<8> g0 = lds_g8(reinterpret_cast<const G*>(st + o) + tt);
-                    float dq = 0.0f;
+                if (MODE) {
+                    const FVec<8> g0 = lds_g8(reinterpret_cast<const G*>(st + o) + tt); o += L::kGb;
+                    if (DOT) {
+                        float dq = 0.0f;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) dq = fmaf(g0.x[i], gg.x[i], dq);
-                    accd += (double)dq;
+                        for (int i = 0; i < 8; ++i) dq = fmaf(g0.x[i], gg.x[i], dq);
+                        accd += (double)dq;
+                    }
+                    if (REPLAY) {
+                        const FVec<8> g1 = lds_g8(reinterpret_cast<const G*>(st + o) + tt);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            advance_moments_elem(mm.x[i], vv.x[i], __fmul_rn(g0.x[i], gs0), p);
+                            advance_moments_elem(mm.x[i], vv.x[i], __fmul_rn(g1.x[i], gs1), p);
+                        }
+                    }
                 }
                 const int e = j * L::kElems + tt;
                 if (U.snap) st_f(U.snap + e, th);
@@ -443,6 +512,7 @@ step_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restric
         if (!alive) break;
         const int done = U.full_tiles * L::kElems;
         if (done < U.len) {
+            if (REPLAY) consumer_replay<G, true>(U.m + done, U.v + done, U.g0 + done, U.g1 + done, U.len - done, p, gs0, gs1);
             step_chunk_vec<ADAMW, G, 8>(U.out + done, U.in + done, U.snap ? U.snap + done : nullptr, ADAMW ? U.m + done : nullptr,
                                         ADAMW ? U.v + done : nullptr, U.g + done, U.len - done, p, gscale, acc, U.wb ? U.wb + done : nullptr);
             if (DOT) consumer_dot(U.g0 + done, U.g + done, U.len - done, accd);

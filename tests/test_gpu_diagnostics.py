@@ -178,6 +178,7 @@ def test_long_list_diagnostics_in_the_default_launch_configuration():
         ctx.bind(ptrs)
         ctx.tune(0, variant, 0)
         ctx.enable_diagnostics(on)
+        ctx.set_gradients_persist(name == "staged")      # not used while diagnostics are on: no effect
         g0, g1 = keep[4], keep[5]
         if name == "staged":
             n_active = 0

@@ -1,7 +1,9 @@
 """Parity at the full sizes of the benchmark configurations, in the launch
 configuration bench.py times (default grid and access width, deferred-state flow:
-gxpo_probe_step_deferred, gxpo_probe_extrapolate, gxpo_slow_step, gxpo_gate_update): the flat 1.54e9-parameter buffer, the Qwen2.5-7B-shaped
-list (7.6e9) and the 64-step gate stream on the Llama-3.1-8B-shaped list (8.0e9).
+gxpo_probe_step_deferred, gxpo_probe_extrapolate, gxpo_slow_step, gxpo_gate_update, with
+gxpo_set_gradients_persist wherever g_slow has a buffer of its own): the flat
+1.54e9-parameter buffer, the Qwen2.5-7B-shaped list (7.6e9) and the 64-step gate stream on
+the Llama-3.1-8B-shaped list (8.0e9).
 
 The update is per-coordinate, so the oracle run on a window of the inputs IS the
 full run restricted to that window: windows are copied to the host before the step
@@ -41,6 +43,7 @@ def _setup(workload, lr, K=5, alpha=0.5):
     cfg, opt = b.make_cfg(K=K, alpha=alpha, lr=lr)
     ctx = b.Context(cfg, opt, b.BF16)
     ctx.bind(ptrs)
+    ctx.set_gradients_persist(not alias)      # as bench.py does: g0 and g1 are buffers nothing overwrites
     return b, ctx, cfg, opt, shapes, desc, alias, d, keep
 
 
