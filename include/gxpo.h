@@ -200,7 +200,8 @@ gxpo_status gxpo_probe_step_deferred(gxpo_ctx* ctx, void* stream);
 
 /* A promise about the caller's gradient buffers, off by default: on != 0 says that g0 and
  * g1 still hold this step's gradients while gxpo_slow_step's sweep runs (nothing reuses
- * them between the backward passes, and g_slow has a buffer of its own).  After
+ * them between the backward passes, and g_slow has a buffer of its own), and that device
+ * scalars given to gxpo_set_grad_scale for them keep their values until then as well.  After
  * gxpo_probe_step_deferred, gxpo_probe_extrapolate may then leave m and v unwritten once
  * more, and the slow step's sweep replays both probe steps' moment updates in registers from
  * g0 and g1 before it takes its own step: 18 + 20 + 30 = 68 instead of 72 bytes per
