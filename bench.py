@@ -4,10 +4,11 @@
 A "step" is one whole active step of Algorithm 1's parameter-space update over
 the workload's tensor list: probe step 0, probe step 1, extrapolate + reposition,
 slow step with the in-sweep norm, gate update.  By default that is 3 sweeps + 1 tiny
-kernel moving 72 bytes per parameter (--flow deferred: the first probe step leaves m, v
-to the fused second-probe + extrapolation sweep); --flow fused moves 84, --flow unfused
-(the four separate calls) 94.  The
-three gradient buffers are synthetic and already resident.
+kernel moving 68 bytes per parameter (--flow deferred: the first probe step and, since
+the benchmark's g0 and g1 buffers stay intact, the fused second-probe + extrapolation
+sweep too leave m, v to the slow step's sweep; 72 with --no-persist); --flow fused moves
+84, --flow unfused (the four separate calls) 94.  The three gradient buffers are
+synthetic and already resident.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 
@@ -61,11 +62,11 @@ def parse_args():
     ap.add_argument("--unit-tiles", type=int, default=0)
     ap.add_argument("--fallback", action="store_true", help="time the single-pass fallback step")
     ap.add_argument("--flow", default="deferred", choices=["deferred", "fused", "unfused"],
-                    help="deferred: probe_step_deferred + probe_extrapolate (72 B/param, default); "
+                    help="deferred: probe_step_deferred + probe_extrapolate (68 B/param on long lists, default); "
                          "fused: probe_step(0) + probe_extrapolate (84); unfused: the four separate sweeps (94)")
     ap.add_argument("--emit-bf16", action="store_true",
                     help="also keep bfloat16 model-weight copies (gxpo_bind_model_weights, bf16-only theta1): "
-                         "16 + 30 + 28 = 74 B/param, and the caller needs no cast sweeps")
+                         "16 + 22 + 32 = 70 B/param, and the caller needs no cast sweeps")
     ap.add_argument("--no-persist", action="store_true",
                     help="do not promise that g0 and g1 outlive the slow step (72 instead of 68 B/param in the deferred flow)")
     ap.add_argument("--diagnostics", action="store_true",
