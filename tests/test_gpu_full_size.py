@@ -100,10 +100,18 @@ def _check_window(keep, lo, hi, st, scale, theta0, theta2, alpha, what, rtol=2e-
     return nsat
 
 
-def _one_active_step_vs_oracle(workload, lr, picks_fn, full_oracle_norm, extra_windows=()):
+def _one_active_step_vs_oracle(workload, lr, picks_fn, full_oracle_norm, extra_windows=(), K=5, emit=False):
     import torch
-    b, ctx, cfg, opt, shapes, desc, alias, d, keep = _setup(workload, lr)
+    b, ctx, cfg, opt, shapes, desc, alias, d, keep = _setup(workload, lr, K=K)
     assert "reduced" not in desc, desc           # the full size is the point of this test
+    weights = None
+    if emit:                                     # bench.py --emit-bf16: bfloat16 copies, theta1 as bfloat16 only
+        weights = torch.full((d,), float("nan"), dtype=torch.bfloat16, device="cuda")
+        offs, acc = [], 0
+        for _, k in shapes:
+            offs.append(acc)
+            acc += k
+        ctx.bind_model_weights([weights.data_ptr() + 2 * o for o in offs], only_bf16_theta1=True)
     gcfg, ocfg = gu.ora_cfgs(cfg, opt)
     wins = _windows(shapes, picks_fn(shapes)) + list(extra_windows)
     before = [_grab(keep, lo, hi) for lo, hi in wins]
@@ -132,8 +140,17 @@ def _one_active_step_vs_oracle(workload, lr, picks_fn, full_oracle_norm, extra_w
                               f"{workload} [{lo},{hi})")
     total = sum(hi - lo for lo, hi in wins)
     assert nsat < 1e-3 * total                    # saturated scale factors are rare
+    if emit:
+        # the copy is the round-to-nearest-even bfloat16 of the float32 point beside it
+        # (the oracle's rounding function applied to the library's own theta)
+        theta = keep[0]
+        for lo, hi in wins:
+            want = ora.round_to_bf16(gu.to_host_f64(theta[lo:hi]))
+            got = weights[lo:hi].view(torch.int16).cpu().numpy().view(np.uint16)
+            ok = (want & 0x7FFF) <= 0x7F80
+            np.testing.assert_array_equal(got[ok], want[ok])
     ctx.close()
-    del keep
+    del keep, weights
     torch.cuda.empty_cache()
 
 
@@ -145,6 +162,21 @@ def test_flat_1p54b_one_active_step(lr):
     def picks(shapes):
         return [(0, "head"), (0, "chunk"), (0, "mid"), (0, "tail")]
     _one_active_step_vs_oracle("flat_1p54b", lr, picks, full_oracle_norm=True)
+
+
+@pytest.mark.parametrize("K", [3, 10])
+def test_flat_1p54b_other_depths(K):
+    """The paper's other virtual depths at full size (K = 5 is the default above)."""
+    def picks(shapes):
+        return [(0, "head"), (0, "chunk"), (0, "tail")]
+    _one_active_step_vs_oracle("flat_1p54b", 1e-3, picks, full_oracle_norm=False, K=K)
+
+
+def test_flat_1p54b_with_bf16_model_weight_copies():
+    """bench.py --emit-bf16 at full size: same float32 results, and the bfloat16 copies."""
+    def picks(shapes):
+        return [(0, "head"), (0, "chunk"), (0, "tail")]
+    _one_active_step_vs_oracle("flat_1p54b", 1e-3, picks, full_oracle_norm=False, emit=True)
 
 
 def test_flat_2p5b_offsets_beyond_two_to_the_31():
@@ -251,7 +283,8 @@ def test_llama31_8b_list_64_step_gate_stream():
     # both paths were timed (milliseconds per step, steady state)
     act = float(np.median(t_active[3:40])) if len(t_active) > 43 else float(np.median(t_active[3:]))
     fb = float(np.median(t_fallback[1:]))
-    print(f"\nllama31_8b d={d}: active step {act:.1f} ms ({72 * d / act / 1e6:.0f} GB/s), "
+    per_param = 72 if alias else 68              # the promise is used where g_slow has its own buffer
+    print(f"\nllama31_8b d={d}: active step {act:.1f} ms ({per_param * d / act / 1e6:.0f} GB/s), "
           f"fallback step {fb:.1f} ms ({26 * d / fb / 1e6:.0f} GB/s), g_slow aliases g0: {alias}")
     assert fb < act
     ctx.close()
