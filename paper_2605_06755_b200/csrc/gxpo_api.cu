@@ -823,7 +823,7 @@ gxpo_status gxpo_slow_step(gxpo_ctx* c, void* stream) {
     c->state_lag = 0;
     if (want_dot && !dot_inside) {
         const bool bf16 = c->grad_dtype == GXPO_BF16;
-        long long g = (long long)c->sm_count * 8;        // 64 warps per SM, one chunk each at a time
+        long long g = (long long)c->sm_count * 4;        // what fits at 64 registers: 32 warps per SM, one chunk each at a time
         if (g * (kThreads / 32) > c->num_chunks) g = (c->num_chunks + kThreads / 32 - 1) / (kThreads / 32);
         if (bf16) dot_kernel<uint16_t><<<(int)g, kThreads, 0, (cudaStream_t)stream>>>(c->d_descs, c->d_chunks, c->num_chunks, 0, 2, c->d_partials, c->d_ticket, c->d_diag + kDiagN);
         else      dot_kernel<float><<<(int)g, kThreads, 0, (cudaStream_t)stream>>>(c->d_descs, c->d_chunks, c->num_chunks, 0, 2, c->d_partials, c->d_ticket, c->d_diag + kDiagN);
@@ -892,7 +892,7 @@ gxpo_status gxpo_clip_grad_norm(gxpo_ctx* c, int which, double max_norm, void* s
     if (!ok) return fail(c, GXPO_ERR_STATE, "clip the gradient right before the sweep that consumes it");
     cudaStream_t s = (cudaStream_t)stream;
     if (c->num_chunks > 0) {
-        long long g = (long long)c->sm_count * 8;        // 64 warps per SM, one chunk each at a time
+        long long g = (long long)c->sm_count * 4;        // what fits at 64 registers: 32 warps per SM, one chunk each at a time
         if (g * (kThreads / 32) > c->num_chunks) g = (c->num_chunks + kThreads / 32 - 1) / (kThreads / 32);
         if (c->grad_dtype == GXPO_BF16)
             dot_kernel<uint16_t><<<(int)g, kThreads, 0, s>>>(c->d_descs, c->d_chunks, c->num_chunks, which, which, c->d_partials, c->d_ticket, c->d_gnorm + which);
