@@ -69,6 +69,9 @@ def parse_args():
                          "16 + 22 + 32 = 70 B/param, and the caller needs no cast sweeps")
     ap.add_argument("--no-persist", action="store_true",
                     help="do not promise that g0 and g1 outlive the slow step (72 instead of 68 B/param in the deferred flow)")
+    ap.add_argument("--clip", type=float, default=0.0,
+                    help="global-norm clipping of every gradient at this value (gxpo_clip_grad_norm: one 2 B/param "
+                         "norm pass per gradient, the coefficient applied inside the sweeps); 0 = off")
     ap.add_argument("--diagnostics", action="store_true",
                     help="gather the per-step diagnostics too (adds a 4 B/param <g0, g_slow> pass after the slow step)")
     ap.add_argument("--no-e2e", action="store_true")
@@ -338,32 +341,43 @@ def run_ours(args):
              "unfused": ["probe_step0", "probe_step1", "extrapolate", "slow_step"]}[flow]
     if args.fallback:
         names = ["fallback_step"]
+    # the calls behind the names, in order; with --clip a norm pass goes in front of each
+    # sweep that consumes a new gradient (the recipe's global-norm clipping)
+    calls = {"fallback_step": lambda: ctx.probe_step(-1, stream),
+             "probe_step0_deferred": lambda: ctx.probe_step_deferred(stream),
+             "probe_step0": lambda: ctx.probe_step(0, stream),
+             "probe_step1": lambda: ctx.probe_step(1, stream),
+             "extrapolate": lambda: ctx.extrapolate(stream),
+             "probe_extrapolate": lambda: ctx.probe_extrapolate(stream),
+             "probe_extrapolate_deferred": lambda: ctx.probe_extrapolate(stream),
+             "probe_extrapolate_nostate": lambda: ctx.probe_extrapolate(stream),
+             "slow_step": lambda: ctx.slow_step(stream),
+             "slow_step_replay": lambda: ctx.slow_step(stream)}
+    clip = float(getattr(args, "clip", 0.0) or 0.0)
+    if clip > 0.0:
+        consumes = {"fallback_step": 0, "probe_step0_deferred": 0, "probe_step0": 0, "probe_step1": 1,
+                    "probe_extrapolate": 1, "probe_extrapolate_deferred": 1, "probe_extrapolate_nostate": 1,
+                    "slow_step": 2, "slow_step_replay": 2}
+        with_clip = []
+        for nm in names:
+            if nm in consumes:
+                k = consumes[nm]
+                cn = f"clip_norm_g{k}"
+                calls[cn] = (lambda k=k: ctx.clip_grad_norm(k, clip, stream))
+                with_clip.append(cn)
+            with_clip.append(nm)
+        names = with_clip
     n_ev = len(names) + 1
 
     def one_step(evs=None):
-        def mark(i):
+        if evs:
+            evs[0].record(stream)
+        for i, nm in enumerate(names):
+            calls[nm]()
             if evs:
-                evs[i].record(stream)
-        mark(0)
+                evs[i + 1].record(stream)
         if args.fallback:
-            ctx.probe_step(-1, stream)
-            mark(1)
             return None
-        if flow == "deferred":
-            ctx.probe_step_deferred(stream)
-        else:
-            ctx.probe_step(0, stream)
-        mark(1)
-        if flow != "unfused":
-            ctx.probe_extrapolate(stream)
-            mark(2)
-        else:
-            ctx.probe_step(1, stream)
-            mark(2)
-            ctx.extrapolate(stream)
-            mark(3)
-        ctx.slow_step(stream)
-        mark(n_ev - 1)
         if world > 1:
             dist.all_reduce(sumsq)        # the one exchange of a sharded step: 8 bytes
         return ctx.gate_update(stream, allow_nonfinite=True)
@@ -414,6 +428,9 @@ def run_ours(args):
         alg_bytes["probe_extrapolate_deferred"] += 2
         alg_bytes["slow_step"] += 2
     kernel_of = dict(KERNEL_OF)
+    for k in range(3):
+        alg_bytes[f"clip_norm_g{k}"] = 2
+        kernel_of[f"clip_norm_g{k}"] = "dot_kernel"
     alg_bytes["probe_extrapolate_nostate"] = alg_bytes["probe_extrapolate_deferred"] - 8   # m, v not written
     alg_bytes["slow_step_replay"] = alg_bytes["slow_step"] + 4              # g0 and g1 read once more
     if diag and not alias:      # <g0, g_slow>, timed with the slow step: g0 read once more inside the staged
@@ -461,7 +478,8 @@ def run_ours(args):
                                 "active (probe with deferred state, probe+extrapolate in one sweep, slow step, gate)",
                     "fused": "active (probe, probe+extrapolate in one sweep, slow step, gate)",
                     "unfused": "active (probe, probe, extrapolate, slow step, gate)"}[flow],
-                   "bf16_model_weight_copies": emit, "diagnostics": diag, "gradients_persist": persist, "g_slow_aliases_g0": alias, "l2": "inputs larger than L2 (no flush needed)",
+                   "bf16_model_weight_copies": emit, "diagnostics": diag, "gradients_persist": persist,
+                   "clip_grad_norm": clip if clip > 0.0 else None, "g_slow_aliases_g0": alias, "l2": "inputs larger than L2 (no flush needed)",
                    "parallelism": f"dp{world} (independent shards, one 8-byte all-reduce per step)" if world > 1 else "1 GPU"},
         "hbm_gbs_whole_step": whole_gbs, "hbm_frac_whole_step": whole_gbs / peak,
         "hbm_frac_of_8tbs_nominal": whole_gbs / 8000.0,
