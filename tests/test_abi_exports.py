@@ -62,3 +62,20 @@ def test_header_is_c99_and_a_plain_c_program_links_against_the_library(tmp_path)
                            str(src), "-o", str(exe), lib, "-Wl,-rpath," + os.path.dirname(lib)])
     out = subprocess.check_output([str(exe)]).decode().split()
     assert out == ["20", "2147483648"]
+
+
+def test_readme_c_example_compiles_against_the_header(tmp_path):
+    """The C snippet in README.md is the call sequence users copy: it must compile as C99
+    against include/gxpo.h (compile only; running it needs a GPU and gradients)."""
+    import re
+    import subprocess
+    text = open(os.path.join(ROOT, "README.md")).read()
+    snippet = re.search(r"```c\n(.*?)```", text, re.S).group(1)
+    assert "gxpo_probe_step_deferred" in snippet and "gxpo_set_gradients_persist" in snippet
+    src = tmp_path / "readme.c"
+    src.write_text('#include "gxpo.h"\n'
+                   "int one_training_run(const gxpo_tensor* tensors, int n_tensors, void* stream) {\n"
+                   + snippet + "    return 0;\n}\n")
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-Wno-unused-variable",
+                           "-Wno-unused-but-set-variable", "-I", os.path.join(ROOT, "include"), "-c", str(src),
+                           "-o", str(tmp_path / "readme.o")])
