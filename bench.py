@@ -334,7 +334,8 @@ def run_ours(args):
     flow = args.flow
     n_chunks = sum((k + 32767) // 32768 for _, k in shapes)
     staged = args.variant == 3 or (args.variant == 0 and n_chunks >= 32 * props.multi_processor_count)
-    lag = persist and staged and not diag     # the fused sweep leaves m, v unwritten; the slow sweep replays from g0, g1
+    # the fused sweep leaves m, v unwritten and the slow sweep replays them from g0, g1 (both staged, from 8 chunks per SM on)
+    lag = persist and not diag and (args.variant == 3 or (args.variant == 0 and n_chunks >= 8 * props.multi_processor_count))
     names = {"deferred": (["probe_step0_deferred", "probe_extrapolate_nostate", "slow_step_replay"] if lag else
                           ["probe_step0_deferred", "probe_extrapolate_deferred", "slow_step"]),
              "fused": ["probe_step0", "probe_extrapolate", "slow_step"],
@@ -436,11 +437,12 @@ def run_ours(args):
     if diag and not alias:      # <g0, g_slow>, timed with the slow step: g0 read once more inside the staged
         alg_bytes["slow_step"] += 2 if staged else 4      # sweep (already there when it replays), else a pass
                                                           # of its own over both gradients
+    kernel_of["probe_extrapolate_nostate"] = "fused_bulk_light_kernel"
+    kernel_of["slow_step_replay"] = "step_bulk_kernel"
     if staged:
         # the fused sweep runs in its bulk-copy staged kernel (the library's default for long lists)
         kernel_of["probe_extrapolate"] = kernel_of["probe_extrapolate_deferred"] = "fused_bulk_kernel"
-        kernel_of["probe_extrapolate_nostate"] = "fused_bulk_light_kernel"
-        kernel_of["slow_step_replay"] = "step_bulk_kernel"
+
         for nm in ("probe_step0", "probe_step1", "slow_step", "fallback_step"):   # AdamW sweeps that write m, v back
             kernel_of[nm] = "step_bulk_kernel"
     kernels = {nm: {"kernel": kernel_of[nm], "ms": ms, "bytes_per_param": alg_bytes[nm],

@@ -206,9 +206,9 @@ gxpo_status gxpo_probe_step_deferred(gxpo_ctx* ctx, void* stream);
  * more, and the slow step's sweep replays both probe steps' moment updates in registers from
  * g0 and g1 before it takes its own step: 18 + 20 + 30 = 68 instead of 72 bytes per
  * parameter, bit-identical theta, m and v.  The library uses this where it pays (AdamW on
- * lists long enough for the shared-memory staged sweep, see gxpo_tune, with diagnostics
- * off) and never when some tensor's g_slow pointer equals its g0 or g1 pointer; elsewhere
- * the promise changes nothing.  Between gxpo_probe_extrapolate and gxpo_slow_step m and v in memory are then
+ * lists of at least 8 chunks of 32768 parameters per SM, with diagnostics off and
+ * gxpo_tune's variant 0 or 3) and never when some tensor's g_slow pointer equals its g0 or
+ * g1 pointer; elsewhere the promise changes nothing.  Between gxpo_probe_extrapolate and gxpo_slow_step m and v in memory are then
  * two steps behind; a caller who breaks the promise gets wrong moments, not an error.
  * Paper: no counterpart (Algorithm 1 does not say where the optimizer state lives between
  * its three steps).  Errors: STATE mid-step. */
