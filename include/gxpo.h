@@ -208,8 +208,9 @@ gxpo_status gxpo_probe_step_deferred(gxpo_ctx* ctx, void* stream);
  * parameter, bit-identical theta, m and v.  The library uses this where it pays (AdamW on
  * lists of at least 8 chunks of 32768 parameters per SM, with diagnostics off and
  * gxpo_tune's variant 0 or 3) and never when some tensor's g_slow pointer equals its g0 or
- * g1 pointer; elsewhere the promise changes nothing.  Between gxpo_probe_extrapolate and gxpo_slow_step m and v in memory are then
- * two steps behind; a caller who breaks the promise gets wrong moments, not an error.
+ * g1 pointer; elsewhere the promise changes nothing.  Between gxpo_probe_extrapolate and
+ * gxpo_slow_step m and v in memory are then two steps behind; a caller who breaks the
+ * promise gets wrong moments, not an error.
  * Paper: no counterpart (Algorithm 1 does not say where the optimizer state lives between
  * its three steps).  Errors: STATE mid-step. */
 gxpo_status gxpo_set_gradients_persist(gxpo_ctx* ctx, int on);
