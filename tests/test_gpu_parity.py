@@ -406,15 +406,19 @@ def test_fused_call_order():
 
 @pytest.mark.parametrize("flow", ["deferred", "fused", "unfused", "fallback"])
 @pytest.mark.parametrize("placement", [0, 1])
-def test_no_sweep_writes_outside_its_tensors(flow, placement):
+@pytest.mark.parametrize("staging", ["registers", "staged", "staged+promise"])
+def test_no_sweep_writes_outside_its_tensors(flow, placement, staging):
     """Every output buffer (theta, work, m, v and the bfloat16 copies) sits between two
     guard bands filled with a sentinel; after a step the bands must be untouched and the
-    read-only gradient buffers bit-identical.  Sizes end mid-vector, mid-tile and
-    mid-chunk, aligned and misaligned."""
+    read-only gradient buffers bit-identical.  Sizes end mid-vector, mid-tile, mid-stage and
+    mid-chunk, aligned and misaligned; the shared-memory staged sweeps (with and without the
+    gradients-persist promise, which needs diagnostics off) are held to the same."""
     import torch
+    if staging == "staged+promise" and flow != "deferred":
+        pytest.skip("the promise only matters in the deferred flow")
     b = _binding()
-    sizes = [1, 7, 2049, 32768 + 3, 2 * 32768 - 1, 70001]
-    offsets = [0, 3, 0, 0, 1, 0]
+    sizes = [1, 7, 2049, 32768 + 3, 2 * 32768 - 1, 70001, 3 * 4096 + 2048 + 5]
+    offsets = [0, 3, 0, 0, 1, 0, 0]
     GUARD = 4096
     sentinel = 1234.5
 
@@ -439,7 +443,9 @@ def test_no_sweep_writes_outside_its_tensors(flow, placement):
     ctx, cfg, opt = _ctx(b, "bf16", lr=1e-3, K=5, alpha=0.5, placement=placement)
     ctx.bind(ptrs)
     ctx.bind_model_weights(wptrs)
-    ctx.enable_diagnostics(True)
+    ctx.tune(0, 2 if staging == "registers" else 3, 0)
+    ctx.enable_diagnostics(staging != "staged+promise")
+    ctx.set_gradients_persist(staging == "staged+promise")
     for _ in range(2):
         if flow == "fallback":
             ctx.probe_step(-1)
