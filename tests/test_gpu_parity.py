@@ -247,19 +247,31 @@ def test_access_variants_and_launch_shapes_agree_bitwise():
         assert o[3] == pytest.approx(outs[0][3], rel=1e-7)
 
 
-def test_run_to_run_determinism():
+@pytest.mark.parametrize("staged", [False, True])
+def test_run_to_run_determinism(staged):
+    """Two runs on the same bits give the same bits, the norm included: the reductions have a
+    fixed order for a fixed launch shape (register-staged sweeps; and the shared-memory
+    staged ones under the gradients-persist promise, diagnostics included in a second step)."""
     b = _binding()
-    n = 3 * 32768 + 11
+    n = 5 * 32768 + 4096 + 11
     got = []
     for _ in range(2):
         pr = _problem(n, seed=5, grad_dtype="bf16")
         ctx, cfg, opt = _ctx(b, "bf16", lr=1e-3)
         ctx.bind([pr.ptrs()])
-        res = ctx.active_step(allow_nonfinite=True)
-        got.append((gu.to_host_f64(pr.theta), res.norm))
+        if staged:
+            ctx.tune(0, 3, 0)
+            ctx.set_gradients_persist(True)
+        res = ctx.active_step(allow_nonfinite=True, deferred=staged)
+        ctx.enable_diagnostics(True)
+        res2 = ctx.active_step(allow_nonfinite=True, deferred=staged)
+        d = ctx.get_diagnostics()
+        got.append((gu.to_host_f64(pr.theta), gu.to_host_f64(pr.m), res.norm, res2.norm,
+                    (d.g0_norm, d.g1_norm, d.cos_g0_gslow, d.ratio_mean, d.ratio_std, d.scale_mean, d.disp_ratio)))
         ctx.close()
     np.testing.assert_array_equal(got[0][0], got[1][0])
-    assert got[0][1] == got[1][1]                       # bitwise: fixed summation order
+    np.testing.assert_array_equal(got[0][1], got[1][1])
+    assert got[0][2:] == got[1][2:]                     # bitwise: fixed summation order
 
 
 def test_probe_step_against_library_adamw_on_device():
