@@ -416,9 +416,9 @@ def test_fused_call_order():
     ctx.close()
 
 
-@pytest.mark.parametrize("flow", ["deferred", "fused", "unfused", "fallback"])
+@pytest.mark.parametrize("flow,staging", [(f, s) for f in ("deferred", "fused", "unfused", "fallback")
+                                          for s in ("registers", "staged")] + [("deferred", "staged+promise")])
 @pytest.mark.parametrize("placement", [0, 1])
-@pytest.mark.parametrize("staging", ["registers", "staged", "staged+promise"])
 def test_no_sweep_writes_outside_its_tensors(flow, placement, staging):
     """Every output buffer (theta, work, m, v and the bfloat16 copies) sits between two
     guard bands filled with a sentinel; after a step the bands must be untouched and the
@@ -426,8 +426,6 @@ def test_no_sweep_writes_outside_its_tensors(flow, placement, staging):
     mid-chunk, aligned and misaligned; the shared-memory staged sweeps (with and without the
     gradients-persist promise, which needs diagnostics off) are held to the same."""
     import torch
-    if staging == "staged+promise" and flow != "deferred":
-        pytest.skip("the promise only matters in the deferred flow")
     b = _binding()
     sizes = [1, 7, 2049, 32768 + 3, 2 * 32768 - 1, 70001, 3 * 4096 + 2048 + 5]
     offsets = [0, 3, 0, 0, 1, 0, 0]
