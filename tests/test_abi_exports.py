@@ -55,6 +55,7 @@ def test_header_is_c99_and_a_plain_c_program_links_against_the_library(tmp_path)
         "    if (c.K != 5 || o.kind != GXPO_OPT_ADAMW) return 2;\n"
         '    if (strcmp(gxpo_status_string(GXPO_ERR_TIMEOUT), "device-side wait timed out") != 0) return 3;\n'
         "    if (gxpo_probe_step(NULL, 0, NULL) != GXPO_ERR_INVALID_ARG) return 4;\n"
+        "    if (gxpo_set_gradients_persist(NULL, 1) != GXPO_ERR_INVALID_ARG) return 5;\n"
         '    printf("%d %lld\\n", c.window, (long long)GXPO_NOALLOC_MAX_PARAMS);\n'
         "    return 0;\n}\n")
     exe = tmp_path / "use"
