@@ -13,6 +13,10 @@ synthetic and already resident.
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 
 prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+With --gpus N > 1 every GPU runs the step on a list of its own (the update shards without
+any exchange but the 8-byte sum behind the gate).  Under a launcher that has set
+WORLD_SIZE (torch.distributed.run) this process is one of its ranks; without one it starts
+the N ranks itself, one process per GPU.
 """
 from __future__ import annotations
 
@@ -300,9 +304,12 @@ def run_ours(args):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but {world} rank(s) are running")
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        world = dist.get_world_size()        # what the communicator really spans
     props = torch.cuda.get_device_properties(local)
     stream = torch.cuda.current_stream()
 
@@ -623,11 +630,80 @@ def run_surrogate(args):
     print(json.dumps(line), flush=True)
 
 
+# ----------------------------------------------------------------------------
+# several GPUs: one process per GPU
+# ----------------------------------------------------------------------------
+def rank_environment(rank, world, port, base=None):
+    """Environment of one rank: what torch.distributed.run would set for a single node."""
+    env = dict(os.environ if base is None else base)
+    env.update({"RANK": str(rank), "LOCAL_RANK": str(rank), "WORLD_SIZE": str(world),
+                "LOCAL_WORLD_SIZE": str(world), "MASTER_ADDR": "127.0.0.1", "MASTER_PORT": str(port)})
+    return env
+
+
+def free_port():
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def spawn_ranks(world, cmd, poll_s=0.2):
+    """Start `cmd` once per rank (ranks 0..world-1, LOCAL_RANK = RANK, one node, rendezvous on
+    127.0.0.1) and wait for all of them.  Every rank inherits stdout and stderr, so rank 0's one
+    JSON line and the communication library's own log reach the caller untouched.  When a rank
+    fails the others are terminated (exactly the processes started here).  Returns the list of
+    exit codes."""
+    port = free_port()
+    procs = [subprocess.Popen(cmd, env=rank_environment(r, world, port)) for r in range(world)]
+    codes = [None] * world
+    failed = False
+    while any(c is None for c in codes):
+        for r, p in enumerate(procs):
+            if codes[r] is None:
+                codes[r] = p.poll()
+                if codes[r] not in (None, 0):
+                    failed = True
+        if failed:
+            for r, p in enumerate(procs):
+                if codes[r] is None:
+                    p.terminate()
+            for r, p in enumerate(procs):
+                if codes[r] is None:
+                    try:
+                        codes[r] = p.wait(timeout=30)
+                    except subprocess.TimeoutExpired:
+                        p.kill()
+                        codes[r] = p.wait()
+            break
+        time.sleep(poll_s)
+    return codes
+
+
 def main():
     args = parse_args()
+    if args.gpus < 1:
+        raise SystemExit("--gpus must be >= 1")
     if args.impl == "reference":
         run_reference(args)
-    elif args.workload == "surrogate_1e8":
+        return
+    launched = "WORLD_SIZE" in os.environ
+    if launched and int(os.environ["WORLD_SIZE"]) != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} contradicts WORLD_SIZE={os.environ['WORLD_SIZE']} of the launcher")
+    if args.gpus > 1 and args.workload == "surrogate_1e8":
+        raise SystemExit("the surrogate workload is a one-GPU harness")
+    if args.gpus > 1 and not launched:
+        # no launcher around us: be the launcher
+        import torch
+        have = torch.cuda.device_count()
+        if have < args.gpus:
+            raise SystemExit(f"--gpus {args.gpus} but only {have} CUDA device(s) are visible")
+        codes = spawn_ranks(args.gpus, [sys.executable, os.path.abspath(__file__)] + sys.argv[1:])
+        bad = [(r, c) for r, c in enumerate(codes) if c != 0]
+        if bad:
+            raise SystemExit(f"rank(s) failed (rank, exit code): {bad}")
+        return
+    if args.workload == "surrogate_1e8":
         run_surrogate(args)
     else:
         run_ours(args)
