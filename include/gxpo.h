@@ -48,10 +48,13 @@ typedef enum {
     GXPO_ERR_ALIGNMENT = 2,   /* a pointer is not aligned to its element size */
     GXPO_ERR_STATE = 3,       /* call out of order for Algorithm 1, or nothing bound */
     GXPO_ERR_CUDA = 4,        /* a CUDA runtime call failed; see gxpo_last_error */
-    GXPO_ERR_TIMEOUT = 5,     /* a bounded device-side wait gave up (only the bulk-copy staged
-                                 variant of the fused sweep waits on anything; the default
-                                 kernels and all reductions are wait-free); reported by the
-                                 gate update that ends the step */
+    GXPO_ERR_TIMEOUT = 5,     /* a bounded device-side wait gave up (only the shared-memory
+                                 staged sweeps wait on anything; the register-staged kernels
+                                 and all reductions are wait-free).  An active step reports it
+                                 from the gate update that ends the step; a fallback step, which
+                                 has no gate update, from the next gxpo_probe_step /
+                                 gxpo_probe_step_deferred / gxpo_gate_peek / gxpo_gate_last /
+                                 gxpo_state_export on the context, once */
     GXPO_ERR_NONFINITE = 6    /* ||g_slow|| was not finite; the gate was tripped */
 } gxpo_status;
 
@@ -138,8 +141,10 @@ void gxpo_destroy(gxpo_ctx* ctx);
 
 /* Bind a tensor list (count == 1 is the flat-buffer case).  Copies the descriptors
  * and builds the chunk table on the device; the list itself is not kept.  May be
- * called again between steps to re-bind.  Waits for the device before it replaces
- * an earlier table.
+ * called again between steps to re-bind.  Before it overwrites an earlier table it waits
+ * for this context's own outstanding work (the last gate read-back, the last fallback
+ * sweep) and for nothing else: other streams of the process keep running, and no device
+ * memory is freed or allocated unless the new list needs a larger table than any before.
  * Errors: INVALID_ARG (null list entry fields, n < 0, count < 0, m/v missing for
  * AdamW), ALIGNMENT (pointer not aligned to its element size), STATE (mid-step). */
 gxpo_status gxpo_bind(gxpo_ctx* ctx, const gxpo_tensor* list, int count);
@@ -157,7 +162,7 @@ gxpo_status gxpo_bind(gxpo_ctx* ctx, const gxpo_tensor* list, int count);
  * theta^{t,1} (gxpo_probe_extrapolate recomputes the float32 value anyway), so `work` is
  * left untouched; needs PINGPONG placement and a buffer for every non-empty tensor.
  * Pass weights_bf16 = NULL to unbind.  gxpo_bind drops the binding.  Only legal between
- * steps; waits for the device. */
+ * steps; waits for this context's own outstanding work, like gxpo_bind. */
 gxpo_status gxpo_bind_model_weights(gxpo_ctx* ctx, void* const* weights_bf16, int count,
                                     int only_bf16_theta1);
 
@@ -398,8 +403,34 @@ gxpo_status gxpo_slow_step_noalloc(float* theta, float* m, float* v, const void*
  * usable.  Only legal between steps; waits for `stream`. */
 gxpo_status gxpo_selftest_bounded_wait(gxpo_ctx* ctx, void* stream);
 
+/* Host-side fault injection for tests of the error path: sets the device error word on
+ * `stream` exactly as a bounded wait that gave up would, without running any waiting
+ * kernel.  The step in flight (or the next one) then reports GXPO_ERR_TIMEOUT where the
+ * description of that status says.  The context stays usable. */
+gxpo_status gxpo_selftest_inject_timeout(gxpo_ctx* ctx, void* stream);
+
 /* Number of kernels this context has launched so far. */
 long long gxpo_launch_count(const gxpo_ctx* ctx);
+
+/* What the most recent sweep call of this context launched: which kernel function the
+ * library's dispatch chose for the bound list (it depends on the optimizer, the list's
+ * length, gxpo_tune, the gradients-persist promise, diagnostics), its grid, and the bytes
+ * per parameter that sweep has to move -- every operand counted once, bfloat16 copies and
+ * replayed gradients included.  A benchmark reads its roofline's byte count and kernel
+ * name from here instead of repeating the dispatch rules.  extra_launches counts further
+ * kernels the same call launched (the separate <g0, g_slow> pass of the diagnostics, whose
+ * bytes are included; the clipping coefficient kernel).
+ * Paper: no counterpart.  Errors: STATE before the first sweep. */
+typedef struct {
+    char kernel[48];              /* e.g. "step_kernel", "step_bulk_kernel", "fused_bulk_light_kernel" */
+    int staged;                   /* 1: operands staged in shared memory by bulk asynchronous copies */
+    int grid;                     /* CTAs launched (0 where the call does not record it) */
+    int bytes_read_per_param;
+    int bytes_written_per_param;
+    int extra_launches;
+    int valid;
+} gxpo_sweep_info;
+gxpo_status gxpo_last_sweep(const gxpo_ctx* ctx, gxpo_sweep_info* out);
 
 const char* gxpo_last_error(const gxpo_ctx* ctx);
 const char* gxpo_status_string(gxpo_status s);

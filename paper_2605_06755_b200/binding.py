@@ -61,6 +61,12 @@ class Diagnostics(ctypes.Structure):
                [(k, ctypes.c_longlong) for k in ("n", "n_active", "n_irregular")]
 
 
+class SweepInfo(ctypes.Structure):
+    _fields_ = [("kernel", ctypes.c_char * 48), ("staged", ctypes.c_int), ("grid", ctypes.c_int),
+                ("bytes_read_per_param", ctypes.c_int), ("bytes_written_per_param", ctypes.c_int),
+                ("extra_launches", ctypes.c_int), ("valid", ctypes.c_int)]
+
+
 _vp = ctypes.c_void_p
 _sigs = {
     "gxpo_default_cfg": (None, [ctypes.POINTER(Cfg), ctypes.POINTER(OptCfg)]),
@@ -94,7 +100,9 @@ _sigs = {
                                       ctypes.c_longlong, _vp, ctypes.POINTER(GateResult)]),
     "gxpo_tune": (ctypes.c_int, [_vp, ctypes.c_int, ctypes.c_int, ctypes.c_int]),
     "gxpo_selftest_bounded_wait": (ctypes.c_int, [_vp, _vp]),
+    "gxpo_selftest_inject_timeout": (ctypes.c_int, [_vp, _vp]),
     "gxpo_launch_count": (ctypes.c_longlong, [_vp]),
+    "gxpo_last_sweep": (ctypes.c_int, [_vp, ctypes.POINTER(SweepInfo)]),
     "gxpo_last_error": (ctypes.c_char_p, [_vp]),
     "gxpo_status_string": (ctypes.c_char_p, [ctypes.c_int]),
     "gxpo_quad_grad": (ctypes.c_int, [_vp, _vp, _vp, _vp, ctypes.c_longlong, _vp]),
@@ -303,8 +311,16 @@ class Context:
         """Returns the status code (ERR_TIMEOUT is the expected outcome)."""
         return _lib.gxpo_selftest_bounded_wait(self._h, _stream_ptr(stream))
 
+    def selftest_inject_timeout(self, stream=None):
+        self._check(_lib.gxpo_selftest_inject_timeout(self._h, _stream_ptr(stream)))
+
     def launch_count(self) -> int:
         return _lib.gxpo_launch_count(self._h)
+
+    def last_sweep(self) -> SweepInfo:
+        out = SweepInfo()
+        self._check(_lib.gxpo_last_sweep(self._h, ctypes.byref(out)))
+        return out
 
     # -- convenience: the calls of one active step in Algorithm 1's order, for callers
     #    whose three gradient buffers are already filled (benchmarks, replay) --------

@@ -92,6 +92,18 @@ struct gxpo_ctx {
     // host mirror
     long long t, s_star, t_opt;
     long long launches;
+    gxpo_sweep_info last_sweep;        // what the most recent sweep launched (gxpo_last_sweep)
+    int wb_any;                        // some tensor has a bfloat16 model-weight copy bound
+    // waiting for this context's own work only (re-binding, checkpointing)
+    cudaStream_t copy_stream;          // non-blocking; table uploads and state copies
+    cudaEvent_t idle_event;            // recorded after work that no gate update follows
+    int idle_marked;
+    long long desc_cap, chunk_cap;     // capacity of d_descs / d_chunks (entries); tables only grow
+    // device error word after a fallback step (no gate kernel runs there to collect it)
+    int* h_err;                        // pinned
+    cudaEvent_t err_done;
+    int err_pending;
+    long long err_step;
     const void* occ_key[32];           // resident CTAs per SM, per kernel (cache)
     int occ_val[32];
     int occ_n;
@@ -119,6 +131,27 @@ gxpo_status fail(gxpo_ctx* c, gxpo_status s, const char* fmt, ...) {
     } while (0)
 
 bool finite_f(float x) { return std::isfinite(x); }
+
+// Remember that `s` carries work of this context which no gate update will follow (a fallback
+// step, a clipping pass between steps), so that wait_idle can wait for exactly that work.
+gxpo_status mark_idle_work(gxpo_ctx* c, cudaStream_t s) {
+    CUDA_TRY(c, cudaEventRecord(c->idle_event, s));
+    c->idle_marked = 1;
+    return GXPO_OK;
+}
+
+// Describe the sweep just launched: kernel function, launch shape and the bytes per parameter
+// it has to move.  bench and tests read this instead of re-deriving the dispatch.
+void note_sweep(gxpo_ctx* c, const char* kernel, int staged, int grid, int rd, int wr) {
+    gxpo_sweep_info& i = c->last_sweep;
+    std::snprintf(i.kernel, sizeof(i.kernel), "%s", kernel);
+    i.staged = staged;
+    i.grid = grid;
+    i.bytes_read_per_param = rd;
+    i.bytes_written_per_param = wr;
+    i.extra_launches = 0;
+    i.valid = 1;
+}
 
 gxpo_status check_cfg(gxpo_ctx* c, const gxpo_cfg* g, const gxpo_opt_cfg* o, int grad_dtype) {
     if (g->K < 2 || g->K > 4096) return fail(c, GXPO_ERR_INVALID_ARG, "K must be in [2, 4096], got %d", g->K);
@@ -207,6 +240,24 @@ StepParams make_step_params(gxpo_ctx* c, int which_grad, int in_sel, int out_sel
     return p;
 }
 
+// Bytes per parameter a sweep has to move (algorithmic: every operand once).
+int grad_bytes(const gxpo_ctx* c) { return c->grad_dtype == GXPO_BF16 ? 2 : 4; }
+void note_step(gxpo_ctx* c, const StepParams& p, bool list, bool staged, int grid, bool dot) {
+    const bool adamw = c->opt.kind == GXPO_OPT_ADAMW;
+    const int G = grad_bytes(c);
+    const int rd = 4 + (adamw ? 8 : 0) + G + (p.replay ? 2 * G : 0) + (dot ? G : 0);
+    const int wr = (p.skip_out ? 0 : 4) + ((adamw && p.write_state) ? 8 : 0) + (p.snapshot ? 4 : 0) +
+                   ((p.emit && list && c->wb_any) ? 2 : 0);
+    note_sweep(c, staged ? "step_bulk_kernel" : "step_kernel", staged ? 1 : 0, grid, rd, wr);
+}
+void note_fused(gxpo_ctx* c, const FusedParams& p, bool list, bool defer, const char* kernel, bool staged, int grid) {
+    const bool adamw = c->opt.kind == GXPO_OPT_ADAMW;
+    const int G = grad_bytes(c);
+    const int rd = (defer ? 4 : 8) + (adamw ? 8 : 0) + 2 * G;
+    const int wr = 4 + ((adamw && p.step.write_state) ? 8 : 0) + ((list && c->wb_any) ? 2 : 0);
+    note_sweep(c, kernel, staged ? 1 : 0, grid, rd, wr);
+}
+
 typedef void (*StepFn)(const TensorDesc*, const ChunkRef*, long long, TensorDesc, StepParams, int,
                        double*, unsigned*, double*);
 typedef void (*ExtrapFn)(const TensorDesc*, const ChunkRef*, long long, TensorDesc, ExtrapParams, int,
@@ -278,6 +329,7 @@ gxpo_status launch_step_bulk_t(gxpo_ctx* c, cudaStream_t s, const TensorDesc* de
                                           c->d_diag_partials, dot_out);
     c->launches += 1;
     CUDA_TRY(c, cudaGetLastError());
+    note_step(c, p, chunks != nullptr, true, (int)g, dot_out != nullptr);
     return GXPO_OK;
 }
 gxpo_status launch_step_bulk(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
@@ -315,6 +367,7 @@ gxpo_status launch_step(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, co
     fn<<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, ush, c->d_partials, c->d_ticket, sumsq);
     c->launches += 1;
     CUDA_TRY(c, cudaGetLastError());
+    note_step(c, p, chunks != nullptr, false, grid, false);
     return GXPO_OK;
 }
 
@@ -330,6 +383,7 @@ gxpo_status launch_extrap(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, 
     fn<<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, ush, c->d_diag_partials, c->d_ticket, c->d_diag);
     c->launches += 1;
     CUDA_TRY(c, cudaGetLastError());
+    note_sweep(c, "extrap_kernel", 0, grid, 8 + 2 * grad_bytes(c), 4 + ((chunks && c->wb_any) ? 2 : 0));
     return GXPO_OK;
 }
 
@@ -342,11 +396,13 @@ gxpo_status launch_bulk_t(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, 
     BulkFn fn = diag ? fused_bulk_kernel<ADAMW, G, DEFER, true> : fused_bulk_kernel<ADAMW, G, DEFER, false>;
     int smem = (int)BulkLayout<ADAMW, G, DEFER>::kTotal;
     int want_per_sm = kDefaultCtasBulk;
+    const char* name = "fused_bulk_kernel";
     if constexpr (ADAMW && DEFER) {
         if (!p.step.write_state && !diag) {   // m and v stay unwritten: the latency-bound shape, two CTAs per SM
             fn = fused_bulk_light_kernel<G>;                      // (with diagnostics it would not fit the registers)
             smem = (int)BulkLayout<true, G, true, true>::kTotal;
             want_per_sm = 2;
+            name = "fused_bulk_light_kernel";
         }
     }
     // first launch of this instantiation in this context: allow the ring's shared memory and
@@ -368,6 +424,7 @@ gxpo_status launch_bulk_t(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, 
                                           c->d_ticket, c->d_diag);
     c->launches += 1;
     CUDA_TRY(c, cudaGetLastError());
+    note_fused(c, p, chunks != nullptr, DEFER, name, true, (int)g);
     return GXPO_OK;
 }
 gxpo_status launch_fused_bulk(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
@@ -403,6 +460,7 @@ gxpo_status launch_fused(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, c
     fn<<<grid, kThreads, 0, s>>>(descs, chunks, num_chunks, flat, p, ush, c->d_diag_partials, c->d_ticket, c->d_diag);
     c->launches += 1;
     CUDA_TRY(c, cudaGetLastError());
+    note_fused(c, p, chunks != nullptr, defer, "fused_kernel", false, grid);
     return GXPO_OK;
 }
 
@@ -452,6 +510,41 @@ gxpo_status finish_gate(gxpo_ctx* c) {
     o.active = r.active; o.tripped = r.tripped; o.t = r.t; o.s_star = r.s_star;
     o.norm = r.norm; o.z = r.z; o.mu = r.mu; o.sigma = r.sigma;
     c->have_gate = 1;
+    return GXPO_OK;
+}
+
+// A fallback step runs no gate kernel, so nothing collects the device error word a bounded
+// wait may have raised in its staged sweep.  The sweep is therefore followed by a 4-byte
+// read-back of the word (and its reset); the next call that looks at the context's state
+// folds it in here and reports the incomplete step once.
+gxpo_status enqueue_error_readback(gxpo_ctx* c, cudaStream_t s, long long step) {
+    CUDA_TRY(c, cudaMemcpyAsync(c->h_err, c->d_err, sizeof(int), cudaMemcpyDeviceToHost, s));
+    CUDA_TRY(c, cudaMemsetAsync(c->d_err, 0, sizeof(int), s));
+    CUDA_TRY(c, cudaEventRecord(c->err_done, s));
+    c->err_pending = 1;
+    c->err_step = step;
+    return GXPO_OK;
+}
+gxpo_status collect_fallback_error(gxpo_ctx* c) {
+    if (!c->err_pending) return GXPO_OK;
+    CUDA_TRY(c, cudaEventSynchronize(c->err_done));
+    c->err_pending = 0;
+    if (*c->h_err) {
+        *c->h_err = 0;
+        return fail(c, GXPO_ERR_TIMEOUT, "a bounded device-side wait gave up during fallback step %lld: its outputs are incomplete", c->err_step);
+    }
+    return GXPO_OK;
+}
+
+// Wait until everything this context has enqueued so far is complete -- its own work only, not
+// the device: a pending gate read-back, then whatever followed the last gate update.
+gxpo_status wait_idle(gxpo_ctx* c) {
+    gxpo_status st = finish_gate(c);
+    if (st != GXPO_OK) return st;
+    if (c->idle_marked) {
+        CUDA_TRY(c, cudaEventSynchronize(c->idle_event));
+        c->idle_marked = 0;
+    }
     return GXPO_OK;
 }
 
@@ -567,6 +660,11 @@ gxpo_status gxpo_create(const gxpo_cfg* cfg, const gxpo_opt_cfg* opt, int grad_d
     if (e == cudaSuccess) e = cudaMalloc(&c->d_result, sizeof(GateResult));
     if (e == cudaSuccess) e = cudaMallocHost(&c->h_result, sizeof(GateResult));
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->gate_done, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->idle_event, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->err_done, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaMallocHost(&c->h_err, sizeof(int));
+    if (e == cudaSuccess) *c->h_err = 0;
     if (e == cudaSuccess) e = cudaMalloc(&c->d_clip, 3 * sizeof(float));
     if (e == cudaSuccess) e = cudaMalloc(&c->d_gnorm, 6 * sizeof(double));
     if (e == cudaSuccess) e = cudaMalloc(&c->d_diag, (kDiagN + 1) * sizeof(double));
@@ -604,6 +702,10 @@ void gxpo_destroy(gxpo_ctx* c) {
     cudaFree(c->d_result);
     if (c->h_result) cudaFreeHost(c->h_result);
     if (c->gate_done) cudaEventDestroy(c->gate_done);
+    if (c->idle_event) cudaEventDestroy(c->idle_event);
+    if (c->err_done) cudaEventDestroy(c->err_done);
+    if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+    if (c->h_err) cudaFreeHost(c->h_err);
     delete c->h_descs;
     cudaFree(c->d_clip);
     cudaFree(c->d_gnorm);
@@ -654,18 +756,26 @@ gxpo_status gxpo_bind(gxpo_ctx* c, const gxpo_tensor* list, int count) {
         const long long nc = (descs[(size_t)i].n + kChunk - 1) / kChunk;
         for (long long k = 0; k < nc; ++k) chunks.push_back(ChunkRef{(unsigned)i, (unsigned)k});
     }
-    CUDA_TRY(c, cudaDeviceSynchronize());
-    cudaFree(c->d_descs); c->d_descs = nullptr;
-    cudaFree(c->d_chunks); c->d_chunks = nullptr;
-    c->num_chunks = 0; c->num_tensors = 0; c->total_params = 0;
-    if (count > 0) {
+    // The old tables may still be read by this context's last sweeps: wait for those (this
+    // context's work only; other streams of the process keep running), then overwrite the
+    // tables in place.  They are reallocated only when the new list needs more room.
+    { gxpo_status ws = wait_idle(c); if (ws != GXPO_OK) return ws; }
+    c->num_chunks = 0; c->num_tensors = 0; c->total_params = 0; c->bound = 0;
+    if ((long long)descs.size() > c->desc_cap) {
+        cudaFree(c->d_descs); c->d_descs = nullptr; c->desc_cap = 0;
         CUDA_TRY(c, cudaMalloc(&c->d_descs, descs.size() * sizeof(TensorDesc)));
-        CUDA_TRY(c, cudaMemcpy(c->d_descs, descs.data(), descs.size() * sizeof(TensorDesc), cudaMemcpyHostToDevice));
+        c->desc_cap = (long long)descs.size();
     }
-    if (!chunks.empty()) {
+    if ((long long)chunks.size() > c->chunk_cap) {
+        cudaFree(c->d_chunks); c->d_chunks = nullptr; c->chunk_cap = 0;
         CUDA_TRY(c, cudaMalloc(&c->d_chunks, chunks.size() * sizeof(ChunkRef)));
-        CUDA_TRY(c, cudaMemcpy(c->d_chunks, chunks.data(), chunks.size() * sizeof(ChunkRef), cudaMemcpyHostToDevice));
+        c->chunk_cap = (long long)chunks.size();
     }
+    if (count > 0)
+        CUDA_TRY(c, cudaMemcpyAsync(c->d_descs, descs.data(), descs.size() * sizeof(TensorDesc), cudaMemcpyHostToDevice, c->copy_stream));
+    if (!chunks.empty())
+        CUDA_TRY(c, cudaMemcpyAsync(c->d_chunks, chunks.data(), chunks.size() * sizeof(ChunkRef), cudaMemcpyHostToDevice, c->copy_stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->copy_stream));
     c->num_chunks = (long long)chunks.size();
     c->num_tensors = count;
     c->total_params = total;
@@ -674,6 +784,7 @@ gxpo_status gxpo_bind(gxpo_ctx* c, const gxpo_tensor* list, int count) {
     c->state_lag = 0;
     c->diag_ready = 0;
     c->only_bf16_theta1 = 0;
+    c->wb_any = 0;
     if (!c->h_descs) c->h_descs = new (std::nothrow) std::vector<TensorDesc>();
     if (!c->h_descs) return fail(c, GXPO_ERR_INVALID_ARG, "out of host memory");
     *c->h_descs = descs;
@@ -696,11 +807,17 @@ gxpo_status gxpo_bind_model_weights(gxpo_ctx* c, void* const* weights_bf16, int 
     }
     if (only_bf16_theta1 && (!all || c->cfg.placement != GXPO_PLACE_PINGPONG))
         return fail(c, GXPO_ERR_INVALID_ARG, "only_bf16_theta1 needs a bfloat16 buffer for every tensor and PINGPONG placement");
-    for (size_t i = 0; i < descs.size(); ++i)
+    int any = 0;
+    for (size_t i = 0; i < descs.size(); ++i) {
         descs[i].wb = static_cast<uint16_t*>(weights_bf16 ? weights_bf16[i] : nullptr);
-    CUDA_TRY(c, cudaDeviceSynchronize());
-    if (!descs.empty())
-        CUDA_TRY(c, cudaMemcpy(c->d_descs, descs.data(), descs.size() * sizeof(TensorDesc), cudaMemcpyHostToDevice));
+        if (descs[i].wb && descs[i].n > 0) any = 1;
+    }
+    { gxpo_status ws = wait_idle(c); if (ws != GXPO_OK) return ws; }
+    if (!descs.empty()) {
+        CUDA_TRY(c, cudaMemcpyAsync(c->d_descs, descs.data(), descs.size() * sizeof(TensorDesc), cudaMemcpyHostToDevice, c->copy_stream));
+        CUDA_TRY(c, cudaStreamSynchronize(c->copy_stream));
+    }
+    c->wb_any = any;
     c->only_bf16_theta1 = only_bf16_theta1 ? 1 : 0;
     return GXPO_OK;
 }
@@ -714,16 +831,25 @@ gxpo_status gxpo_probe_step(gxpo_ctx* c, int which, void* stream) {
     const int place = c->cfg.placement;
     if (which == -1) {
         if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "fallback step in the middle of an active step");
+        { gxpo_status fe = collect_fallback_error(c); if (fe != GXPO_OK) return fe; }
         c->t_opt += 1;
         StepParams p = make_step_params(c, 0, 0, 0, 0, 0);
         gxpo_status st = launch_step(c, s, c->d_descs, c->d_chunks, c->num_chunks, none, p, c->d_sumsq);
         if (st != GXPO_OK) { c->t_opt -= 1; return st; }
+        // only the staged sweep waits on anything; it alone can raise the error word
+        if (c->num_chunks > 0 && step_runs_staged(c, p, c->num_chunks)) {
+            st = enqueue_error_readback(c, s, c->t);
+            if (st != GXPO_OK) return st;
+        }
+        st = mark_idle_work(c, s);
+        if (st != GXPO_OK) return st;
         c->t += 1;
         expire_clips(c);
         return GXPO_OK;
     }
     if (which == 0) {
         if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "probe step 0 must start a step");
+        { gxpo_status fe = collect_fallback_error(c); if (fe != GXPO_OK) return fe; }
         { gxpo_status fg = finish_gate(c); if (fg != GXPO_OK) return fg; }
         if (!gate_active(c)) return fail(c, GXPO_ERR_STATE, "gate has tripped (s*=%lld, t=%lld): only fallback steps are legal", c->s_star, c->t);
         c->t_opt += 1;
@@ -750,6 +876,7 @@ gxpo_status gxpo_probe_step_deferred(gxpo_ctx* c, void* stream) {
     if (!c) return GXPO_ERR_INVALID_ARG;
     if (!c->bound) return fail(c, GXPO_ERR_STATE, "nothing bound: call gxpo_bind first");
     if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "probe step 0 must start a step");
+    { gxpo_status fe = collect_fallback_error(c); if (fe != GXPO_OK) return fe; }
     { gxpo_status fg = finish_gate(c); if (fg != GXPO_OK) return fg; }
     if (!gate_active(c)) return fail(c, GXPO_ERR_STATE, "gate has tripped (s*=%lld, t=%lld): only fallback steps are legal", c->s_star, c->t);
     const TensorDesc none = {};
@@ -833,6 +960,8 @@ gxpo_status gxpo_slow_step(gxpo_ctx* c, void* stream) {
         else      dot_kernel<float><<<(int)g, kThreads, 0, (cudaStream_t)stream>>>(c->d_descs, c->d_chunks, c->num_chunks, 0, 2, c->d_partials, c->d_ticket, c->d_diag + kDiagN);
         c->launches += 1;
         CUDA_TRY(c, cudaGetLastError());
+        c->last_sweep.bytes_read_per_param += 2 * grad_bytes(c);   // the extra pass reads g0 and g_slow
+        c->last_sweep.extra_launches = 1;
     }
     c->phase = SLOW_DONE;
     return GXPO_OK;
@@ -860,6 +989,7 @@ gxpo_status gxpo_gate_update_async(gxpo_ctx* c, void* stream) {
 
 gxpo_status gxpo_gate_last(gxpo_ctx* c, gxpo_gate_result* out) {
     if (!c) return GXPO_ERR_INVALID_ARG;
+    { gxpo_status fe = collect_fallback_error(c); if (fe != GXPO_OK) return fe; }
     gxpo_status st = finish_gate(c);
     if (st != GXPO_OK) return st;
     if (!c->have_gate) return fail(c, GXPO_ERR_STATE, "no gate update has run yet");
@@ -910,6 +1040,9 @@ gxpo_status gxpo_clip_grad_norm(gxpo_ctx* c, int which, double max_norm, void* s
     clip_coef_kernel<<<1, 32, 0, s>>>(c->d_gnorm + which, max_norm, c->d_clip + which, c->d_gnorm + 3 + which);
     c->launches += 1;
     CUDA_TRY(c, cudaGetLastError());
+    note_sweep(c, "dot_kernel", 0, 0, grad_bytes(c), 0);
+    c->last_sweep.extra_launches = 1;                       // the coefficient kernel
+    if (c->phase == IDLE) { gxpo_status ms = mark_idle_work(c, s); if (ms != GXPO_OK) return ms; }
     c->gscale[which] = c->d_clip + which;
     return GXPO_OK;
 }
@@ -964,8 +1097,23 @@ gxpo_status gxpo_selftest_bounded_wait(gxpo_ctx* c, void* stream) {
     return GXPO_OK;
 }
 
+gxpo_status gxpo_selftest_inject_timeout(gxpo_ctx* c, void* stream) {
+    if (!c) return GXPO_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    CUDA_TRY(c, cudaMemsetAsync(c->d_err, 1, sizeof(int), s));      // any non-zero word means "a wait gave up"
+    return GXPO_OK;
+}
+
+gxpo_status gxpo_last_sweep(const gxpo_ctx* c, gxpo_sweep_info* out) {
+    if (!c || !out) return GXPO_ERR_INVALID_ARG;
+    if (!c->last_sweep.valid) return fail(const_cast<gxpo_ctx*>(c), GXPO_ERR_STATE, "no sweep has been launched yet");
+    *out = c->last_sweep;
+    return GXPO_OK;
+}
+
 gxpo_status gxpo_gate_peek(const gxpo_ctx* c, int* active, long long* s_star, long long* t) {
     if (!c) return GXPO_ERR_INVALID_ARG;
+    { gxpo_status fe = collect_fallback_error(const_cast<gxpo_ctx*>(c)); if (fe != GXPO_OK) return fe; }
     { gxpo_status fg = finish_gate(const_cast<gxpo_ctx*>(c)); if (fg != GXPO_OK) return fg; }
     if (active) *active = gate_active(c) ? 1 : 0;
     if (s_star) *s_star = c->s_star;
@@ -1030,16 +1178,18 @@ gxpo_status gxpo_state_export(gxpo_ctx* c, void* buf, size_t* len) {
     if (!buf) { *len = need; return GXPO_OK; }
     if (*len < need) { *len = need; return fail(c, GXPO_ERR_INVALID_ARG, "buffer too small: need %zu bytes", need); }
     if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "state export in the middle of a step");
-    { gxpo_status fg = finish_gate(c); if (fg != GXPO_OK) return fg; }
-    CUDA_TRY(c, cudaDeviceSynchronize());
+    { gxpo_status fe = collect_fallback_error(c); if (fe != GXPO_OK) return fe; }
+    { gxpo_status ws = wait_idle(c); if (ws != GXPO_OK) return ws; }
     GateState g;
-    CUDA_TRY(c, cudaMemcpy(&g, c->d_gate, sizeof(g), cudaMemcpyDeviceToHost));
+    CUDA_TRY(c, cudaMemcpyAsync(&g, c->d_gate, sizeof(g), cudaMemcpyDeviceToHost, c->copy_stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->copy_stream));
     StateHeader h;
     std::memset(&h, 0, sizeof(h));
     h.magic = kMagic; h.version = 1; h.window = c->cfg.window; h.head = g.head; h.count = g.count;
     h.t = c->t; h.s_star = c->s_star; h.t_opt = c->t_opt;
     std::memcpy(buf, &h, sizeof(h));
-    CUDA_TRY(c, cudaMemcpy(static_cast<char*>(buf) + sizeof(h), c->d_ring, (size_t)c->cfg.window * sizeof(double), cudaMemcpyDeviceToHost));
+    CUDA_TRY(c, cudaMemcpyAsync(static_cast<char*>(buf) + sizeof(h), c->d_ring, (size_t)c->cfg.window * sizeof(double), cudaMemcpyDeviceToHost, c->copy_stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->copy_stream));
     *len = need;
     return GXPO_OK;
 }
@@ -1056,11 +1206,12 @@ gxpo_status gxpo_state_import(gxpo_ctx* c, const void* buf, size_t len) {
     if (h.window != c->cfg.window) return fail(c, GXPO_ERR_INVALID_ARG, "window mismatch: blob %d, context %d", h.window, c->cfg.window);
     if (h.head < 0 || h.head >= h.window || h.count < 0 || h.count > h.window || h.t < 0 || h.t_opt < 0 || h.s_star < -1)
         return fail(c, GXPO_ERR_INVALID_ARG, "corrupt state blob");
-    CUDA_TRY(c, cudaDeviceSynchronize());
+    { gxpo_status ws = wait_idle(c); if (ws != GXPO_OK) return ws; }
     GateState g;
     g.head = h.head; g.count = h.count; g.s_star = h.s_star;
-    CUDA_TRY(c, cudaMemcpy(c->d_gate, &g, sizeof(g), cudaMemcpyHostToDevice));
-    CUDA_TRY(c, cudaMemcpy(c->d_ring, static_cast<const char*>(buf) + sizeof(h), (size_t)c->cfg.window * sizeof(double), cudaMemcpyHostToDevice));
+    CUDA_TRY(c, cudaMemcpyAsync(c->d_gate, &g, sizeof(g), cudaMemcpyHostToDevice, c->copy_stream));
+    CUDA_TRY(c, cudaMemcpyAsync(c->d_ring, static_cast<const char*>(buf) + sizeof(h), (size_t)c->cfg.window * sizeof(double), cudaMemcpyHostToDevice, c->copy_stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->copy_stream));
     c->t = h.t; c->s_star = h.s_star; c->t_opt = h.t_opt;
     return GXPO_OK;
 }
@@ -1160,7 +1311,9 @@ gxpo_status gxpo_step_host(gxpo_ctx* c, const gxpo_tensor* list, int count, long
         out->active = 0; out->tripped = 0; out->t = c->t; out->s_star = c->s_star;
         out->norm = out->z = out->mu = out->sigma = std::nan("");
     }
-    return GXPO_OK;
+    // no gate kernel ran: collect the error word of the staged sweeps here
+    { gxpo_status es = enqueue_error_readback(c, st.stream[0], c->t - 1); if (es != GXPO_OK) return es; }
+    return collect_fallback_error(c);
 }
 
 // ---- surrogate harness ---------------------------------------------------------

@@ -34,13 +34,18 @@ def ulp32(x):
     return np.spacing(np.abs(np.asarray(x, dtype=np.float64)).astype(np.float32)).astype(np.float64)
 
 
-def displacement_slack(theta0, theta2, scale, alpha, ulps=4.0):
+def displacement_slack(theta0, theta2, scale, alpha, ulps=4.0, theta1=None):
     """Absolute slack for outputs that contain (theta2 - theta0) * scale when theta2
     itself was produced by an earlier float32 call: theta2 carries up to a couple of
     ulps of its own rounding, the subtraction cancels the leading digits, and the
     scale factor multiplies what is left.  This is the conditioning of the formula,
-    not an error of either implementation."""
+    not an error of either implementation.  The ulp is that of the largest point on
+    the way: where a step is as large as the parameter itself, theta1 can be several
+    times larger than both theta0 and theta2, and its rounding (at its own magnitude)
+    is what theta2 inherits -- pass theta1 where such coordinates occur."""
     big = np.maximum(np.abs(theta0), np.abs(theta2))
+    if theta1 is not None:
+        big = np.maximum(big, np.abs(theta1))
     with np.errstate(invalid="ignore", over="ignore"):
         return ulps * ulp32(big) * abs(alpha) * np.abs(scale)
 

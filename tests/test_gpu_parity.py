@@ -522,3 +522,138 @@ def test_bounded_wait_gives_up_and_reports_timeout():
     ctx.tune(0, 3, 0)
     assert ctx.active_step(allow_nonfinite=True, deferred=True).t == 2
     ctx.close()
+
+
+def test_injected_timeout_is_reported_by_active_and_by_fallback_steps():
+    """The device error word, raised from the host exactly as a wait that gave up would
+    raise it (no waiting kernel runs): an active step reports it from its gate update; a
+    fallback step, which has no gate update, from the next call that looks at the context.
+    Either way it is reported once and the context stays usable."""
+    b = _binding()
+    pr = _problem(3 * 32768 + 100, 5, "bf16")
+    ctx, cfg, opt = _ctx(b, "bf16", lr=1e-3)
+    ctx.bind([pr.ptrs()])
+    ctx.tune(0, 3, 0)                                        # the staged sweeps: the ones that wait
+    # active step
+    ctx.probe_step_deferred()
+    ctx.selftest_inject_timeout()
+    ctx.probe_extrapolate()
+    ctx.slow_step()
+    with pytest.raises(b.GxpoError) as e:
+        ctx.gate_update()
+    assert e.value.status == b.ERR_TIMEOUT and "step 0" in str(e.value)
+    assert ctx.active_step(deferred=True).t == 2             # reported once; the word was cleared
+    # fallback step
+    ctx.selftest_inject_timeout()
+    ctx.probe_step(-1)                                       # the sweep itself returns OK (asynchronous)
+    with pytest.raises(b.GxpoError) as e:
+        ctx.gate_peek()
+    assert e.value.status == b.ERR_TIMEOUT and "fallback step 2" in str(e.value)
+    assert ctx.gate_peek()[2] == 3                           # once
+    ctx.probe_step(-1)
+    ctx.selftest_inject_timeout()
+    ctx.probe_step(-1)
+    with pytest.raises(b.GxpoError) as e:
+        ctx.probe_step(-1)                                   # the next step refuses to build on an incomplete one
+    assert e.value.status == b.ERR_TIMEOUT and "fallback step 4" in str(e.value)
+    ctx.probe_step(-1)
+    assert ctx.gate_peek()[2] == 6 and ctx.optimizer_steps() == 6 + 4
+    ctx.close()
+
+
+@pytest.mark.parametrize("n", [40003, 3 * 32768 + 5])
+@pytest.mark.parametrize("kind,grad_dtype", [("adamw", "bf16"), ("adamw", "f32"), ("gd", "f32")])
+@pytest.mark.parametrize("mode", ["plain", "staged", "replay"])
+def test_slow_step_call_alone(n, kind, grad_dtype, mode):
+    """Strict 1e-6 check of gxpo_slow_step by itself: the oracle's OptimStep starts from the
+    very bits the library holds before the call (theta-tilde, m, v copied back), so no
+    earlier call's rounding enters and no slack is needed.  `replay`: under the
+    gradients-persist promise m and v in memory still predate the two probe steps and the
+    slow sweep advances them with g0 and g1 first; the oracle is given the same inputs."""
+    if kind == "gd" and mode == "replay":
+        pytest.skip("plain gradient descent has no state to replay")
+    b = _binding()
+    pr = _problem(n, seed=700 + n, grad_dtype=grad_dtype, zero_frac=0.03)
+    ctx, cfg, opt = _ctx(b, grad_dtype, kind=b.OPT_ADAMW if kind == "adamw" else b.OPT_GD, lr=1e-3, K=5, alpha=0.5)
+    gcfg, ocfg = gu.ora_cfgs(cfg, opt)
+    ctx.bind([pr.ptrs()])
+    ctx.tune(0, 0 if mode == "plain" else 3, 0)
+    ctx.set_gradients_persist(mode == "replay")
+    ctx.probe_step_deferred()
+    ctx.probe_extrapolate()
+    grads = pr.oracle_grads()
+    st = ora.State(gu.to_host_f64(pr.theta), ocfg, None if kind == "gd" else gu.to_host_f64(pr.m),
+                   None if kind == "gd" else gu.to_host_f64(pr.v), t_opt=0 if mode == "replay" else 2)
+    if mode == "replay":
+        assert ctx.last_sweep().bytes_written_per_param == 4         # m, v really were left unwritten
+        tilde = st.theta.copy()
+        st.optim_step(grads[0], True)                                # only m, v matter here
+        st.optim_step(grads[1], True)
+        st.theta = tilde
+    with np.errstate(all="ignore"):
+        st.optim_step(grads[2], True)
+    ctx.slow_step()
+    res = ctx.gate_update(allow_nonfinite=True)
+    gu.assert_close(gu.to_host_f64(pr.theta), st.theta, "theta after the slow step alone")
+    if kind == "adamw":
+        gu.assert_close(gu.to_host_f64(pr.m), st.m, "m")
+        gu.assert_close(gu.to_host_f64(pr.v), st.v, "v")
+    assert res.norm == pytest.approx(ora.l2norm(grads[2]), rel=gu.RTOL_NORM)
+    ctx.close()
+
+
+def test_last_sweep_reports_what_the_dispatch_chose():
+    """gxpo_last_sweep is where a benchmark gets kernel names and byte counts from; check it
+    against the documented dispatch on a short list (register-staged), with the staged
+    kernels forced, with bfloat16 copies, and for plain gradient descent."""
+    import torch
+    b = _binding()
+    pr = _problem(3 * 32768 + 5, 9, "bf16")
+    ctx, cfg, opt = _ctx(b, "bf16", lr=1e-3)
+    with pytest.raises(b.GxpoError) as e:
+        ctx.last_sweep()
+    assert e.value.status == b.ERR_STATE
+    ctx.bind([pr.ptrs()])
+
+    def sweep():
+        k = ctx.last_sweep()
+        return k.kernel.decode(), k.staged, k.bytes_read_per_param, k.bytes_written_per_param
+
+    ctx.probe_step(0); assert sweep() == ("step_kernel", 0, 14, 12)
+    ctx.probe_step(1); assert sweep() == ("step_kernel", 0, 14, 12)
+    ctx.extrapolate(); assert sweep() == ("extrap_kernel", 0, 12, 4)
+    ctx.slow_step(); assert sweep() == ("step_kernel", 0, 14, 12)
+    ctx.gate_update(allow_nonfinite=True)
+    ctx.probe_step_deferred(); assert sweep() == ("step_kernel", 0, 14, 4)
+    ctx.probe_extrapolate(); assert sweep() == ("fused_kernel", 0, 16, 12)
+    ctx.slow_step(); ctx.gate_update(allow_nonfinite=True)
+    ctx.probe_step(0); ctx.probe_extrapolate(); assert sweep() == ("fused_kernel", 0, 20, 12)
+    ctx.slow_step(); ctx.gate_update(allow_nonfinite=True)
+    ctx.tune(0, 3, 0)
+    ctx.set_gradients_persist(True)
+    ctx.probe_step_deferred(); assert sweep() == ("step_kernel", 0, 14, 4)
+    ctx.probe_extrapolate(); assert sweep() == ("fused_bulk_light_kernel", 1, 16, 4)
+    ctx.slow_step(); assert sweep() == ("step_bulk_kernel", 1, 18, 12)
+    ctx.gate_update(allow_nonfinite=True)
+    ctx.set_gradients_persist(False)
+    wb = torch.zeros(pr.n, dtype=torch.bfloat16, device="cuda")
+    ctx.bind_model_weights([wb.data_ptr()], only_bf16_theta1=True)
+    ctx.probe_step_deferred(); assert sweep() == ("step_kernel", 0, 14, 2)
+    ctx.probe_extrapolate(); assert sweep() == ("fused_bulk_kernel", 1, 16, 14)
+    ctx.slow_step(); assert sweep() == ("step_bulk_kernel", 1, 14, 14)
+    ctx.gate_update(allow_nonfinite=True)
+    ctx.probe_step(-1); assert sweep() == ("step_bulk_kernel", 1, 14, 14)
+    ctx.clip_grad_norm(0, 1.0); assert sweep() == ("dot_kernel", 0, 2, 0)
+    ctx.close()
+    th, m, v, g0, g1, gs = workloads.llm_inputs_numpy(50000, 3, "f32")
+    pg = gu.Problem(th, None, None, g0, g1, gs)
+    cfg, opt = b.make_cfg(kind=b.OPT_GD, lr=1e-2)
+    gd = b.Context(cfg, opt, b.F32)
+    gd.bind([pg.ptrs()])
+    gd.probe_step(0)
+    k = gd.last_sweep()
+    assert (k.kernel, k.bytes_read_per_param, k.bytes_written_per_param) == (b"step_kernel", 8, 4)
+    gd.probe_extrapolate()
+    k = gd.last_sweep()
+    assert (k.kernel, k.bytes_read_per_param, k.bytes_written_per_param) == (b"fused_kernel", 16, 4)
+    gd.close()

@@ -81,3 +81,76 @@ def test_noalloc_rejects_oversize_and_handles_empty():
     b.slow_step_noalloc(0, 0, 0, 0, 0, b.F32, opt, 1, sumsq.data_ptr())
     torch.cuda.synchronize()
     assert float(sumsq.item()) == 0.0
+
+
+def _oracle_slow_step(th, m, v, gs, ocfg, t_opt):
+    """OptimStep(theta, g_slow) and sum(g_slow^2) by the CPU oracle, on the same bits."""
+    from oracle import gxpo_oracle as ora
+    g = gu.grad_to_f64(gs)
+    st = ora.State(th, ocfg, m, v, t_opt=t_opt - 1)          # optim_step counts this step itself
+    st.optim_step(g, True)
+    return st, ora.sum_squares(g)
+
+
+def _prepare(b, n, seed, grad_dtype, t_opt, what=""):
+    """Seeded inputs on the device; returns (launch(stream), check())."""
+    import torch
+    th, m, v, _, _, gs = workloads.llm_inputs_numpy(n, seed, grad_dtype, warm_state=True)
+    cfg, opt = b.make_cfg(lr=1e-3)
+    _, ocfg = gu.ora_cfgs(cfg, opt)
+    d_th, d_m, d_v = gu.to_dev(th), gu.to_dev(m), gu.to_dev(v)
+    d_gs = gu.to_dev(gs, grad_dtype == "bf16")
+    sumsq = torch.full((1,), float("nan"), dtype=torch.float64, device="cuda")
+
+    def launch(stream=None):
+        b.slow_step_noalloc(d_th.data_ptr(), d_m.data_ptr(), d_v.data_ptr(), d_gs.data_ptr(), n,
+                            b.BF16 if grad_dtype == "bf16" else b.F32, opt, t_opt, sumsq.data_ptr(), stream)
+
+    def check():
+        _compare(d_th, d_m, d_v, sumsq, _oracle_slow_step(th, m, v, gs, ocfg, t_opt), what)
+
+    return launch, check
+
+
+def _compare(d_th, d_m, d_v, sumsq, want, what):
+    st, want_sumsq = want
+    gu.assert_close(gu.to_host_f64(d_th), st.theta, what + " theta")      # one call, the oracle on the same bits: 1e-6
+    gu.assert_close(gu.to_host_f64(d_m), st.m, what + " m")
+    gu.assert_close(gu.to_host_f64(d_v), st.v, what + " v")
+    assert float(sumsq.item()) == pytest.approx(want_sumsq, rel=gu.RTOL_NORM)
+
+
+def test_noalloc_against_the_oracle_with_more_chunks_than_ctas_then_fewer():
+    """700 chunks and a ragged tail: every CTA of the grid takes several chunks in turn, so the
+    per-chunk reduction inside the loop and the reuse of its shared scratch are exercised.
+    Then a much shorter buffer, whose call finds the long call's partial sums still sitting
+    in the slots beyond its own chunks and must not pick them up; then a single parameter.
+    All three against the CPU oracle directly."""
+    import torch
+    b = _binding()
+    for n, seed in ((700 * 32768 + 5, 31), (3 * 32768 + 11, 32), (1, 33)):
+        launch, check = _prepare(b, n, seed, "bf16", t_opt=7, what=f"n={n}")
+        launch()
+        torch.cuda.synchronize()
+        check()
+
+
+def test_noalloc_calls_on_two_streams_ordered_by_an_event():
+    """All calls share the one built-in scratch array, so calls on different streams have to
+    be ordered by the caller.  With an event between them the second call, on another
+    stream, must give the oracle's result just like the first."""
+    import torch
+    b = _binding()
+    launch1, check1 = _prepare(b, 600 * 32768 + 123, 41, "f32", t_opt=3, what="stream 1")
+    launch2, check2 = _prepare(b, 9 * 32768 + 1, 42, "f32", t_opt=4, what="stream 2")
+    torch.cuda.synchronize()                                  # inputs in place; from here on only the event orders
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    launch1(s1)
+    done = torch.cuda.Event()
+    done.record(s1)
+    s2.wait_event(done)                                       # the second call starts after the first has finished
+    launch2(s2)
+    s1.synchronize()
+    s2.synchronize()
+    check1()
+    check2()
