@@ -236,6 +236,7 @@ StepParams make_step_params(gxpo_ctx* c, int which_grad, int in_sel, int out_sel
         p.decay = (float)(1.0 - lr * o.weight_decay);
         p.step_size = (float)(lr / (1.0 - std::pow(b1, t)));
         p.inv_sqrt_bc2 = (float)(1.0 / std::sqrt(1.0 - std::pow(b2, t)));
+        p.den_floor_ok = (p.eps >= 0x1p-120f && p.inv_sqrt_bc2 >= 0.0f) ? 1 : 0;
     }
     return p;
 }
@@ -296,8 +297,18 @@ FusedFn pick_fused(bool adamw, bool bf16, int variant, bool defer, bool diag) {
 }
 
 // The bulk-copy staged AdamW sweep: one CTA per SM, whole chunks.
-typedef void (*StepBulkFn)(const TensorDesc*, const ChunkRef*, long long, TensorDesc, StepParams, double*,
+typedef void (*StepBulkFn)(const TensorDesc*, const ChunkRef*, long long, TensorDesc, StepParams, int, double*,
                            unsigned*, double*, int*, double*, double*);
+
+// Work unit of a staged sweep: whole chunks on long lists; half or quarter chunks (still whole
+// stages) when whole chunks would give a CTA fewer than 32 turns, so that the last round of
+// the round-robin leaves few CTAs idle.
+int bulk_unit_shift(const gxpo_ctx* c, long long num_chunks, long long grid) {
+    if (c->unit_shift >= 0) return c->unit_shift < 2 ? c->unit_shift : 2;
+    int sh = 0;
+    while (sh < 2 && (num_chunks << sh) < 32 * grid) ++sh;
+    return sh;
+}
 template <typename G>
 gxpo_status launch_step_bulk_t(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
                                long long num_chunks, const TensorDesc& flat, const StepParams& p, double* sumsq,
@@ -323,9 +334,10 @@ gxpo_status launch_step_bulk_t(gxpo_ctx* c, cudaStream_t s, const TensorDesc* de
     int per_sm = c->ctas_per_sm > 0 ? c->ctas_per_sm : kDefaultCtasBulk;
     if (per_sm > resident) per_sm = resident;
     long long g = (long long)c->sm_count * per_sm;
-    if (g > num_chunks) g = num_chunks;
+    const int ush = bulk_unit_shift(c, num_chunks, g);
+    if (g > (num_chunks << ush)) g = num_chunks << ush;
     // the diagnostics' partial-sum array is idle between the extrapolation sweep and the next step
-    fn<<<(int)g, kBulkThreads, smem, s>>>(descs, chunks, num_chunks, flat, p, c->d_partials, c->d_ticket, sumsq, c->d_err,
+    fn<<<(int)g, kBulkThreads, smem, s>>>(descs, chunks, num_chunks, flat, p, ush, c->d_partials, c->d_ticket, sumsq, c->d_err,
                                           c->d_diag_partials, dot_out);
     c->launches += 1;
     CUDA_TRY(c, cudaGetLastError());
@@ -388,7 +400,7 @@ gxpo_status launch_extrap(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, 
 }
 
 // The bulk-copy staged variant of the fused sweep: one CTA per SM, whole chunks.
-typedef void (*BulkFn)(const TensorDesc*, const ChunkRef*, long long, TensorDesc, FusedParams, int*, double*,
+typedef void (*BulkFn)(const TensorDesc*, const ChunkRef*, long long, TensorDesc, FusedParams, int, int*, double*,
                        unsigned*, double*);
 template <bool ADAMW, typename G, bool DEFER>
 gxpo_status launch_bulk_t(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, const ChunkRef* chunks,
@@ -419,8 +431,9 @@ gxpo_status launch_bulk_t(gxpo_ctx* c, cudaStream_t s, const TensorDesc* descs, 
     int per_sm = c->ctas_per_sm > 0 ? c->ctas_per_sm : want_per_sm;
     if (per_sm > resident) per_sm = resident;
     long long g = (long long)c->sm_count * per_sm;
-    if (g > num_chunks) g = num_chunks;
-    fn<<<(int)g, kBulkThreads, smem, s>>>(descs, chunks, num_chunks, flat, p, c->d_err, c->d_diag_partials,
+    const int ush = bulk_unit_shift(c, num_chunks, g);
+    if (g > (num_chunks << ush)) g = num_chunks << ush;
+    fn<<<(int)g, kBulkThreads, smem, s>>>(descs, chunks, num_chunks, flat, p, ush, c->d_err, c->d_diag_partials,
                                           c->d_ticket, c->d_diag);
     c->launches += 1;
     CUDA_TRY(c, cudaGetLastError());
@@ -470,6 +483,7 @@ ExtrapParams make_extrap_params(const gxpo_ctx* c, int placement) {
     p.alpha = c->cfg.alpha;
     p.delta = c->cfg.delta;
     p.den_eps = c->cfg.den_eps;
+    p.b_floor_ok = (c->cfg.delta >= 0x1p-120f) ? 1 : 0;
     p.gscale0 = c->gscale[0];
     p.gscale1 = c->gscale[1];
     if (placement == GXPO_PLACE_PINGPONG) { p.theta2_sel = 1; p.theta0_sel = 0; }

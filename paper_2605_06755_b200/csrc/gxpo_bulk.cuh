@@ -83,19 +83,24 @@ template <typename G> struct FusedUnit {
     bool vec;
 };
 
+// Work unit u = piece `u mod 2^unit_shift` of chunk `u >> unit_shift` (whole, half or quarter chunks:
+// always a whole number of stages).  Short lists are dealt in smaller units so that the last
+// round of the round-robin leaves few CTAs idle.
 template <bool ADAMW, typename G, bool DEFER>
-__device__ __forceinline__ bool fused_resolve(long long c, const TensorDesc* descs, const ChunkRef* chunks,
+__device__ __forceinline__ bool fused_resolve(long long u, int unit_shift, const TensorDesc* descs, const ChunkRef* chunks,
                                               const TensorDesc& flat, const FusedParams& p, int stage_elems,
                                               FusedUnit<G>& U) {
+    const long long c = u >> unit_shift;
+    const int unit_len = kChunk >> unit_shift;
     ChunkRef ref;
     TensorDesc d;
     if (chunks) { ref = chunks[c]; d = descs[ref.tensor]; }
     else { ref.tensor = 0; ref.chunk = (unsigned)c; d = flat; }
-    const long long off = (long long)ref.chunk * kChunk;
+    const long long off = (long long)ref.chunk * kChunk + (long long)(u & ((1 << unit_shift) - 1)) * unit_len;
     const long long rem = d.n - off;
     U.len = 0; U.full_tiles = 0; U.vec = false;
     if (rem <= 0) return false;
-    U.len = rem < kChunk ? (int)rem : kChunk;
+    U.len = rem < unit_len ? (int)rem : unit_len;
     U.t1 = (p.step.in_sel ? d.work : d.theta) + off;
     U.t0 = (p.ex.theta0_sel ? d.work : d.theta) + off;
     U.out = d.theta + off;
@@ -144,9 +149,10 @@ struct BulkLayout {
 template <bool ADAMW, typename G, bool DEFER, bool DIAG, bool LIGHT>
 __device__ __forceinline__ void fused_bulk_body(const TensorDesc* __restrict__ descs, const ChunkRef* __restrict__ chunks,
                                                 long long num_chunks, const TensorDesc& flat, const FusedParams& p,
-                                                int* error_word, double* diag_partials, unsigned* ticket,
-                                                double* diag_out) {
+                                                int unit_shift, int* error_word, double* diag_partials,
+                                                unsigned* ticket, double* diag_out) {
     typedef BulkLayout<ADAMW, G, DEFER, LIGHT> L;
+    const long long num_units = num_chunks << unit_shift;
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int kStages = L::kStagesN;
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStages * L::kStage);
@@ -164,9 +170,9 @@ __device__ __forceinline__ void fused_bulk_body(const TensorDesc* __restrict__ d
         if (lane != 0) return;
         unsigned it = 0;
         bool ok = true;
-        for (long long c = blockIdx.x; c < num_chunks && ok; c += gridDim.x) {
+        for (long long u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
             FusedUnit<G> U;
-            if (!fused_resolve<ADAMW, G, DEFER>(c, descs, chunks, flat, p, L::kElems, U)) continue;
+            if (!fused_resolve<ADAMW, G, DEFER>(u, unit_shift, descs, chunks, flat, p, L::kElems, U)) continue;
             for (int j = 0; j < U.full_tiles; ++j, ++it) {
                 const unsigned s = it % kStages, n = it / kStages;
                 // the consumers must have released the stage's previous use
@@ -210,9 +216,9 @@ __device__ __forceinline__ void fused_bulk_body(const TensorDesc* __restrict__ d
     bool alive = true;
     const float gs0 = p.ex.gscale0 ? __ldg(p.ex.gscale0) : 1.0f, gs1 = p.ex.gscale1 ? __ldg(p.ex.gscale1) : 1.0f;
     unsigned it = 0;
-    for (long long c = blockIdx.x; c < num_chunks && alive; c += gridDim.x) {
+    for (long long u = blockIdx.x; u < num_units && alive; u += gridDim.x) {
         FusedUnit<G> U;
-        if (!fused_resolve<ADAMW, G, DEFER>(c, descs, chunks, flat, p, L::kElems, U)) continue;
+        if (!fused_resolve<ADAMW, G, DEFER>(u, unit_shift, descs, chunks, flat, p, L::kElems, U)) continue;
         if (!U.vec) {                                   // misaligned tensor: scalar path, no staging
             for (int e = threadIdx.x; e < U.len; e += kThreads) {
                 float mm = ADAMW ? U.m[e] : 0.0f, vv = ADAMW ? U.v[e] : 0.0f;
@@ -301,9 +307,9 @@ __device__ __forceinline__ void fused_bulk_body(const TensorDesc* __restrict__ d
 template <bool ADAMW, typename G, bool DEFER, bool DIAG>
 __global__ void __launch_bounds__(kBulkThreads, 1)
 fused_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restrict__ chunks,
-                  long long num_chunks, TensorDesc flat, FusedParams p, int* error_word,
+                  long long num_chunks, TensorDesc flat, FusedParams p, int unit_shift, int* error_word,
                   double* diag_partials, unsigned* ticket, double* diag_out) {
-    fused_bulk_body<ADAMW, G, DEFER, DIAG, false>(descs, chunks, num_chunks, flat, p, error_word, diag_partials, ticket, diag_out);
+    fused_bulk_body<ADAMW, G, DEFER, DIAG, false>(descs, chunks, num_chunks, flat, p, unit_shift, error_word, diag_partials, ticket, diag_out);
 }
 
 // The LIGHT shape, two CTAs per SM: 18 warps put 5 on one scheduler, whose 16384 registers
@@ -312,9 +318,9 @@ fused_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restri
 template <typename G>
 __global__ void __launch_bounds__(kBulkThreads, 2)
 fused_bulk_light_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restrict__ chunks,
-                        long long num_chunks, TensorDesc flat, FusedParams p, int* error_word,
+                        long long num_chunks, TensorDesc flat, FusedParams p, int unit_shift, int* error_word,
                         double* diag_partials, unsigned* ticket, double* diag_out) {
-    fused_bulk_body<true, G, true, false, true>(descs, chunks, num_chunks, flat, p, error_word, diag_partials, ticket, diag_out);
+    fused_bulk_body<true, G, true, false, true>(descs, chunks, num_chunks, flat, p, unit_shift, error_word, diag_partials, ticket, diag_out);
 }
 
 // ---------------------------------------------------------------------------
@@ -350,15 +356,17 @@ template <typename G> struct StepUnit {
     int len, full_tiles; bool vec;
 };
 template <bool ADAMW, typename G, int MODE>
-__device__ __forceinline__ bool step_resolve(long long c, const TensorDesc* descs, const ChunkRef* chunks,
+__device__ __forceinline__ bool step_resolve(long long u, int unit_shift, const TensorDesc* descs, const ChunkRef* chunks,
                                              const TensorDesc& flat, const StepParams& p, int stage_elems, StepUnit<G>& U) {
+    const long long c = u >> unit_shift;
+    const int unit_len = kChunk >> unit_shift;
     ChunkRef ref; TensorDesc d;
     if (chunks) { ref = chunks[c]; d = descs[ref.tensor]; } else { ref.tensor = 0; ref.chunk = (unsigned)c; d = flat; }
-    const long long off = (long long)ref.chunk * kChunk;
+    const long long off = (long long)ref.chunk * kChunk + (long long)(u & ((1 << unit_shift) - 1)) * unit_len;
     const long long rem = d.n - off;
     U.len = 0; U.full_tiles = 0; U.vec = false;
     if (rem <= 0) return false;
-    U.len = rem < kChunk ? (int)rem : kChunk;
+    U.len = rem < unit_len ? (int)rem : unit_len;
     U.in = (p.in_sel ? d.work : d.theta) + off;
     U.out = (p.out_sel ? d.work : d.theta) + off;
     U.snap = p.snapshot ? d.work + off : nullptr;
@@ -408,9 +416,10 @@ __device__ __forceinline__ void consumer_replay(float* m, float* v, const G* g0,
 template <bool ADAMW, typename G, int MODE>
 __global__ void __launch_bounds__(kBulkThreads, 1)
 step_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restrict__ chunks,
-                 long long num_chunks, TensorDesc flat, StepParams p, double* partials, unsigned* ticket,
+                 long long num_chunks, TensorDesc flat, StepParams p, int unit_shift, double* partials, unsigned* ticket,
                  double* sumsq_out, int* error_word, double* dot_partials, double* dot_out) {
     typedef StepLayout<ADAMW, G, MODE> L;
+    const long long num_units = num_chunks << unit_shift;
     constexpr bool DOT = (MODE & kStepDot) != 0, REPLAY = (MODE & kStepReplay) != 0;
     constexpr int kStages = kStepStages;
     extern __shared__ __align__(128) unsigned char smem[];
@@ -429,9 +438,9 @@ step_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restric
     if (warp == kConsumerWarps) {
         if (lane != 0) return;
         unsigned it = 0; bool ok = true;
-        for (long long c = blockIdx.x; c < num_chunks && ok; c += gridDim.x) {
+        for (long long u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
             StepUnit<G> U;
-            if (!step_resolve<ADAMW, G, MODE>(c, descs, chunks, flat, p, L::kElems, U)) continue;
+            if (!step_resolve<ADAMW, G, MODE>(u, unit_shift, descs, chunks, flat, p, L::kElems, U)) continue;
             for (int j = 0; j < U.full_tiles; ++j, ++it) {
                 const unsigned s = it % kStages, n = it / kStages;
                 if (n > 0 && !mbar_wait_bounded(empty + s, (n - 1) & 1, stop, kWaitLimit)) { ok = false; break; }
@@ -459,9 +468,9 @@ step_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restric
     const float gs0 = (REPLAY && p.gscale_r0) ? __ldg(p.gscale_r0) : 1.0f;
     const float gs1 = (REPLAY && p.gscale_r1) ? __ldg(p.gscale_r1) : 1.0f;
     double acc = 0.0, accd = 0.0; unsigned it = 0; bool alive = true;
-    for (long long c = blockIdx.x; c < num_chunks && alive; c += gridDim.x) {
+    for (long long u = blockIdx.x; u < num_units && alive; u += gridDim.x) {
         StepUnit<G> U;
-        if (!step_resolve<ADAMW, G, MODE>(c, descs, chunks, flat, p, L::kElems, U)) continue;
+        if (!step_resolve<ADAMW, G, MODE>(u, unit_shift, descs, chunks, flat, p, L::kElems, U)) continue;
         if (!U.vec) {
             if (REPLAY) consumer_replay<G, false>(U.m, U.v, U.g0, U.g1, U.len, p, gs0, gs1);
             step_chunk_scalar<ADAMW, G>(U.out, U.in, U.snap, U.m, U.v, U.g, U.len, p, gscale, acc, U.wb);
