@@ -236,7 +236,6 @@ StepParams make_step_params(gxpo_ctx* c, int which_grad, int in_sel, int out_sel
         p.decay = (float)(1.0 - lr * o.weight_decay);
         p.step_size = (float)(lr / (1.0 - std::pow(b1, t)));
         p.inv_sqrt_bc2 = (float)(1.0 / std::sqrt(1.0 - std::pow(b2, t)));
-        p.den_floor_ok = (p.eps >= 0x1p-120f && p.inv_sqrt_bc2 >= 0.0f) ? 1 : 0;
     }
     return p;
 }
@@ -483,7 +482,6 @@ ExtrapParams make_extrap_params(const gxpo_ctx* c, int placement) {
     p.alpha = c->cfg.alpha;
     p.delta = c->cfg.delta;
     p.den_eps = c->cfg.den_eps;
-    p.b_floor_ok = (c->cfg.delta >= 0x1p-120f) ? 1 : 0;
     p.gscale0 = c->gscale[0];
     p.gscale1 = c->gscale[1];
     if (placement == GXPO_PLACE_PINGPONG) { p.theta2_sel = 1; p.theta0_sel = 0; }
