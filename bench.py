@@ -63,8 +63,9 @@ def parse_args():
                     help="deferred: probe_step_deferred + probe_extrapolate (68 B/param on long lists, default); "
                          "fused: probe_step(0) + probe_extrapolate (84); unfused: the four separate sweeps (94)")
     ap.add_argument("--emit-bf16", action="store_true",
-                    help="also keep bfloat16 model-weight copies (gxpo_bind_model_weights, bf16-only theta1): "
-                         "16 + 22 + 32 = 70 B/param, and the caller needs no cast sweeps")
+                    help="also keep bfloat16 model-weight copies (gxpo_bind_model_weights), so that the caller needs no "
+                         "cast sweeps: theta1 and theta-tilde as bfloat16 only, theta-tilde recomputed by the slow step "
+                         "(16 + 18 + 32 = 66 B/param); with --no-persist only theta1 is bfloat16-only (16 + 30 + 28 = 74)")
     ap.add_argument("--no-persist", action="store_true",
                     help="do not promise that g0 and g1 outlive the slow step (72 instead of 68 B/param in the deferred flow)")
     ap.add_argument("--clip", type=float, default=0.0,
@@ -322,13 +323,16 @@ def run_ours(args):
     # the benchmark's g0 and g1 are buffers of their own that nothing overwrites: say so
     persist = not getattr(args, "no_persist", False) and args.flow == "deferred" and not alias and not args.fallback
     ctx.set_gradients_persist(persist)
+    only16 = False
     if emit:
         weights = torch.empty(d, dtype=torch.bfloat16, device="cuda")
         offs, acc = [], 0
         for _, k in shapes:
             offs.append(acc)
             acc += k
-        ctx.bind_model_weights([weights.data_ptr() + 2 * o for o in offs], only_bf16_theta1=True)
+        only16 = persist and not diag and args.variant in (0, 3)
+        ctx.bind_model_weights([weights.data_ptr() + 2 * o for o in offs],
+                               bf16_only=b.BF16_ONLY_PROBE_POINTS if only16 else b.BF16_ONLY_THETA1)
     if world > 1:
         ctx.set_sumsq_buffer(sumsq.data_ptr())
 
@@ -390,7 +394,9 @@ def run_ours(args):
     relabel = {}
     if "probe_extrapolate_deferred" in sweeps and sweeps["probe_extrapolate_deferred"].kernel == b"fused_bulk_light_kernel":
         relabel["probe_extrapolate_deferred"] = "probe_extrapolate_nostate"      # m, v left unwritten
-    if "slow_step" in sweeps and sweeps["slow_step"].bytes_read_per_param - sweeps["slow_step"].extra_launches * 2 * G == 12 + 3 * G:
+    if "slow_step" in sweeps and sweeps["slow_step"].kernel == b"slow_recompute_bulk_kernel":
+        relabel["slow_step"] = "slow_step_recompute"                             # theta-tilde redone from theta^t, g0, g1
+    elif "slow_step" in sweeps and sweeps["slow_step"].bytes_read_per_param - sweeps["slow_step"].extra_launches * 2 * G == 12 + 3 * G:
         relabel["slow_step"] = "slow_step_replay"                                # g0 and g1 read once more
     lag = bool(relabel)
     for old, new in relabel.items():
@@ -466,7 +472,9 @@ def run_ours(args):
                                 "active (probe with deferred state, probe+extrapolate in one sweep, slow step, gate)",
                     "fused": "active (probe, probe+extrapolate in one sweep, slow step, gate)",
                     "unfused": "active (probe, probe, extrapolate, slow step, gate)"}[flow],
-                   "bf16_model_weight_copies": emit, "diagnostics": diag, "gradients_persist": persist,
+                   "bf16_model_weight_copies": (("theta1 and theta-tilde as bfloat16 only (theta-tilde recomputed by the slow step)"
+                                                 if only16 else "theta1 as bfloat16 only") if emit else False),
+                   "diagnostics": diag, "gradients_persist": persist,
                    "clip_grad_norm": clip if clip > 0.0 else None, "g_slow_aliases_g0": alias, "l2": "inputs larger than L2 (no flush needed)",
                    "parallelism": f"dp{world} (independent shards, one 8-byte all-reduce per step)" if world > 1 else "1 GPU"},
         "hbm_gbs_whole_step": whole_gbs, "hbm_frac_whole_step": whole_gbs / peak,

@@ -101,8 +101,10 @@ typedef struct {
     int placement; /* GXPO_PLACE_* */
 } gxpo_cfg;
 
-/* One parameter tensor.  `work` has the same length as `theta`.  m and v may be
- * NULL for GXPO_OPT_GD.  g0/g1/g_slow are read-only inputs of the context's
+/* One parameter tensor.  `work` has the same length as `theta`; it may be NULL when the
+ * caller only ever takes steps that keep no point there (see gxpo_bind_model_weights:
+ * bfloat16-only probe points; fallback steps), and calls that need it then return
+ * GXPO_ERR_STATE.  m and v may be NULL for GXPO_OPT_GD.  g0/g1/g_slow are read-only inputs of the context's
  * gradient dtype; g_slow may alias g0 or g1 (both are dead once gxpo_extrapolate
  * has run).  No other buffers may overlap. */
 typedef struct {
@@ -158,13 +160,31 @@ gxpo_status gxpo_bind(gxpo_ctx* ctx, const gxpo_tensor* list, int count);
  * (theta^{t+1}) -- then also stores that point rounded to nearest-even bfloat16, which
  * saves the caller a separate cast sweep (read 4 + write 2 bytes per parameter) before
  * each backward pass.  The second probe step's point is never needed and not stored.
- * only_bf16_theta1 != 0: gxpo_probe_step_deferred writes ONLY the bfloat16 copy of
- * theta^{t,1} (gxpo_probe_extrapolate recomputes the float32 value anyway), so `work` is
- * left untouched; needs PINGPONG placement and a buffer for every non-empty tensor.
+ * bf16_only says which float32 points are NOT stored beside their copies:
+ *   GXPO_BF16_BESIDE            every point is stored in float32 and as a copy.
+ *   GXPO_BF16_ONLY_THETA1       gxpo_probe_step_deferred writes ONLY the bfloat16 copy of
+ *                               theta^{t,1} (gxpo_probe_extrapolate recomputes the float32
+ *                               value anyway); `work` is left untouched.
+ *   GXPO_BF16_ONLY_PROBE_POINTS in addition gxpo_probe_extrapolate writes ONLY the bfloat16
+ *                               copy of theta-tilde: theta^t stays in `theta`, m and v stay as
+ *                               they were, and gxpo_slow_step redoes both probe steps and the
+ *                               extrapolation in registers (the same functions on the same
+ *                               bits, hence the float32 theta-tilde whose rounding the third
+ *                               backward pass saw) before its own step.  16 + 18 + 32 = 66
+ *                               bytes per parameter including the three copies, and `work`
+ *                               is never touched: tensors may be bound with work == NULL,
+ *                               20 instead of 24 bytes per parameter resident.  The step must
+ *                               then be gxpo_probe_step_deferred, gxpo_probe_extrapolate,
+ *                               gxpo_slow_step under gxpo_set_gradients_persist(ctx, 1), with
+ *                               AdamW, diagnostics off and g_slow in a buffer of its own;
+ *                               anything else returns GXPO_ERR_STATE before the step starts.
+ * Both ONLY modes need PINGPONG placement and a buffer for every non-empty tensor.
+ * Results (theta, m, v, the copies) are bit-identical across the three modes.
  * Pass weights_bf16 = NULL to unbind.  gxpo_bind drops the binding.  Only legal between
  * steps; waits for this context's own outstanding work, like gxpo_bind. */
+enum { GXPO_BF16_BESIDE = 0, GXPO_BF16_ONLY_THETA1 = 1, GXPO_BF16_ONLY_PROBE_POINTS = 2 };
 gxpo_status gxpo_bind_model_weights(gxpo_ctx* ctx, void* const* weights_bf16, int count,
-                                    int only_bf16_theta1);
+                                    int bf16_only);
 
 /* Algorithm 1, "first/second fast optimizer step" (which = 0, 1) and the fallback
  * phase's single step (which = -1).

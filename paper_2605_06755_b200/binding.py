@@ -26,6 +26,7 @@ OK, ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_STATE, ERR_CUDA, ERR_TIMEOUT, ERR_NONFIN
 OPT_GD, OPT_ADAMW = 0, 1
 F32, BF16 = 0, 1
 PLACE_PINGPONG, PLACE_SNAPSHOT = 0, 1
+BF16_BESIDE, BF16_ONLY_THETA1, BF16_ONLY_PROBE_POINTS = 0, 1, 2
 
 
 class OptCfg(ctypes.Structure):
@@ -209,14 +210,16 @@ class Context:
     def bind(self, tensors: Sequence[TensorPtrs]):
         self._check(_lib.gxpo_bind(self._h, _pack(tensors), len(tensors)))
 
-    def bind_model_weights(self, ptrs, only_bf16_theta1: bool = False):
+    def bind_model_weights(self, ptrs, only_bf16_theta1: bool = False, bf16_only: int = 0):
         """ptrs: device pointers of the bfloat16 copies, one per bound tensor (0 = none),
-        or None to unbind."""
+        or None to unbind.  bf16_only: BF16_BESIDE, BF16_ONLY_THETA1 (also selected by
+        only_bf16_theta1=True) or BF16_ONLY_PROBE_POINTS."""
         if ptrs is None:
             self._check(_lib.gxpo_bind_model_weights(self._h, None, 0, 0))
             return
         arr = (_vp * max(1, len(ptrs)))(*[p or None for p in ptrs])
-        self._check(_lib.gxpo_bind_model_weights(self._h, arr, len(ptrs), 1 if only_bf16_theta1 else 0))
+        mode = int(bf16_only) if bf16_only else (1 if only_bf16_theta1 else 0)
+        self._check(_lib.gxpo_bind_model_weights(self._h, arr, len(ptrs), mode))
 
     def probe_step(self, which: int, stream=None):
         self._check(_lib.gxpo_probe_step(self._h, which, _stream_ptr(stream)))

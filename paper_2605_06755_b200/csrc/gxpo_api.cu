@@ -58,7 +58,10 @@ struct gxpo_ctx {
     int num_tensors;
     int bound;
     std::vector<TensorDesc>* h_descs;  // host copy of the bound descriptors
-    int only_bf16_theta1;              // deferred first probe writes the bfloat16 copy only
+    int only_bf16_theta1;              // GXPO_BF16_ONLY_*: 1 = the deferred first probe writes the bfloat16 copy only;
+                                       // 2 = so does the fused sweep (theta-tilde), and the slow step recomputes it
+    int work_missing;                  // some tensor was bound with work == NULL
+    FusedParams lag_fused;             // mode 2: the fused sweep's parameters, for the recomputing slow step
     long long total_params;
     // reductions and gate
     double* d_partials;
@@ -84,7 +87,8 @@ struct gxpo_ctx {
     int gslow_aliased;                 // some tensor's g_slow shares g0's buffer: no <g0, g_slow>
     int gslow_shares_probe;            // some tensor's g_slow shares g0's or g1's buffer
     int grads_persist;                 // the caller promised that g0 and g1 outlive the slow step's sweep
-    int state_lag;                     // this step's fused sweep left m and v unwritten: the slow step replays
+    int state_lag;                     // this step's fused sweep left m and v unwritten: the slow step replays (1),
+                                       // or recomputes theta-tilde as well (2)
     double* d_diag;                    // kDiagN sums + <g0, g_slow>
     double* d_diag_partials;           // kDiagN x kMaxGrid
     DiagResult* d_diag_result;
@@ -254,7 +258,7 @@ void note_fused(gxpo_ctx* c, const FusedParams& p, bool list, bool defer, const 
     const bool adamw = c->opt.kind == GXPO_OPT_ADAMW;
     const int G = grad_bytes(c);
     const int rd = (defer ? 4 : 8) + (adamw ? 8 : 0) + 2 * G;
-    const int wr = 4 + ((adamw && p.step.write_state) ? 8 : 0) + ((list && c->wb_any) ? 2 : 0);
+    const int wr = (p.step.skip_out ? 0 : 4) + ((adamw && p.step.write_state) ? 8 : 0) + ((list && c->wb_any) ? 2 : 0);
     note_sweep(c, kernel, staged ? 1 : 0, grid, rd, wr);
 }
 
@@ -348,6 +352,45 @@ gxpo_status launch_step_bulk(gxpo_ctx* c, cudaStream_t s, const TensorDesc* desc
                              double* dot_out) {
     return c->grad_dtype == GXPO_BF16 ? launch_step_bulk_t<uint16_t>(c, s, descs, chunks, num_chunks, flat, p, sumsq, dot_out)
                                       : launch_step_bulk_t<float>(c, s, descs, chunks, num_chunks, flat, p, sumsq, dot_out);
+}
+
+// The slow step that recomputes theta-tilde (bfloat16-only probe points): one CTA per SM.
+typedef void (*SlowRecomputeFn)(const TensorDesc*, const ChunkRef*, long long, TensorDesc, FusedParams, StepParams, int,
+                                double*, unsigned*, double*, int*);
+gxpo_status launch_slow_recompute(gxpo_ctx* c, cudaStream_t s, const StepParams& p, double* sumsq) {
+    if (c->num_chunks <= 0) {
+        CUDA_TRY(c, cudaMemsetAsync(sumsq, 0, sizeof(double), s));
+        return GXPO_OK;
+    }
+    const bool bf16 = c->grad_dtype == GXPO_BF16;
+    // one CTA per SM with the replaying sweep's ring; two CTAs with the smaller ring on request (gxpo_tune)
+    const bool two = c->ctas_per_sm == 2;
+    SlowRecomputeFn fn = bf16 ? (two ? slow_recompute_bulk_kernel<uint16_t, 1> : slow_recompute_bulk_kernel<uint16_t, 0>)
+                              : (two ? slow_recompute_bulk_kernel<float, 1> : slow_recompute_bulk_kernel<float, 0>);
+    const int smem = bf16 ? (two ? (int)RecomputeLayout<uint16_t, 1>::kTotal : (int)RecomputeLayout<uint16_t, 0>::kTotal)
+                          : (two ? (int)RecomputeLayout<float, 1>::kTotal : (int)RecomputeLayout<float, 0>::kTotal);
+    int resident = 0;
+    for (int i = 0; i < c->occ_n; ++i)
+        if (c->occ_key[i] == (const void*)fn) resident = c->occ_val[i];
+    if (resident == 0) {
+        CUDA_TRY(c, cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, (const void*)fn, kBulkThreads, (size_t)smem) != cudaSuccess || resident < 1)
+            resident = 1;
+        if (c->occ_n < 32) { c->occ_key[c->occ_n] = (const void*)fn; c->occ_val[c->occ_n] = resident; c->occ_n += 1; }
+    }
+    int per_sm = two ? 2 : 1;
+    if (per_sm > resident) per_sm = resident;
+    long long g = (long long)c->sm_count * per_sm;
+    const int ush = bulk_unit_shift(c, c->num_chunks, g);
+    if (g > (c->num_chunks << ush)) g = c->num_chunks << ush;
+    const TensorDesc none = {};
+    fn<<<(int)g, kBulkThreads, smem, s>>>(c->d_descs, c->d_chunks, c->num_chunks, none, c->lag_fused, p, ush, c->d_partials,
+                                          c->d_ticket, sumsq, c->d_err);
+    c->launches += 1;
+    CUDA_TRY(c, cudaGetLastError());
+    const int G = grad_bytes(c);
+    note_sweep(c, "slow_recompute_bulk_kernel", 1, (int)g, 12 + 3 * G, 12 + ((p.emit && c->wb_any) ? 2 : 0));
+    return GXPO_OK;
 }
 
 // AdamW sweeps that write m and v back run bulk-copy staged on long lists (default) or
@@ -751,10 +794,11 @@ gxpo_status gxpo_bind(gxpo_ctx* c, const gxpo_tensor* list, int count) {
     std::vector<TensorDesc> descs((size_t)count);
     std::vector<ChunkRef> chunks;
     long long total = 0;
-    int aliased = 0, shares_probe = 0;
+    int aliased = 0, shares_probe = 0, work_missing = 0;
     for (int i = 0; i < count; ++i) {
-        gxpo_status s = check_tensor(c, list[i], i, true);
+        gxpo_status s = check_tensor(c, list[i], i, false);
         if (s != GXPO_OK) return s;
+        if (list[i].n > 0 && !list[i].work) work_missing = 1;
         TensorDesc& d = descs[(size_t)i];
         d.theta = list[i].theta; d.work = list[i].work; d.m = list[i].m; d.v = list[i].v;
         d.g[0] = list[i].g0; d.g[1] = list[i].g1; d.g[2] = list[i].g_slow;
@@ -796,6 +840,7 @@ gxpo_status gxpo_bind(gxpo_ctx* c, const gxpo_tensor* list, int count) {
     c->state_lag = 0;
     c->diag_ready = 0;
     c->only_bf16_theta1 = 0;
+    c->work_missing = work_missing;
     c->wb_any = 0;
     if (!c->h_descs) c->h_descs = new (std::nothrow) std::vector<TensorDesc>();
     if (!c->h_descs) return fail(c, GXPO_ERR_INVALID_ARG, "out of host memory");
@@ -817,8 +862,12 @@ gxpo_status gxpo_bind_model_weights(gxpo_ctx* c, void* const* weights_bf16, int 
         if (((uintptr_t)w) & 1u) return fail(c, GXPO_ERR_ALIGNMENT, "tensor %d: bfloat16 pointer is not 2-byte aligned", (int)i);
         if (!w && descs[i].n > 0) all = false;
     }
+    if (only_bf16_theta1 < 0 || only_bf16_theta1 > 2)
+        return fail(c, GXPO_ERR_INVALID_ARG, "bf16_only must be GXPO_BF16_BESIDE (0), GXPO_BF16_ONLY_THETA1 (1) or GXPO_BF16_ONLY_PROBE_POINTS (2)");
     if (only_bf16_theta1 && (!all || c->cfg.placement != GXPO_PLACE_PINGPONG))
-        return fail(c, GXPO_ERR_INVALID_ARG, "only_bf16_theta1 needs a bfloat16 buffer for every tensor and PINGPONG placement");
+        return fail(c, GXPO_ERR_INVALID_ARG, "bfloat16-only points need a bfloat16 buffer for every tensor and PINGPONG placement");
+    if (only_bf16_theta1 == 2 && c->opt.kind != GXPO_OPT_ADAMW)
+        return fail(c, GXPO_ERR_INVALID_ARG, "GXPO_BF16_ONLY_PROBE_POINTS is built for AdamW only");
     int any = 0;
     for (size_t i = 0; i < descs.size(); ++i) {
         descs[i].wb = static_cast<uint16_t*>(weights_bf16 ? weights_bf16[i] : nullptr);
@@ -830,7 +879,7 @@ gxpo_status gxpo_bind_model_weights(gxpo_ctx* c, void* const* weights_bf16, int 
         CUDA_TRY(c, cudaStreamSynchronize(c->copy_stream));
     }
     c->wb_any = any;
-    c->only_bf16_theta1 = only_bf16_theta1 ? 1 : 0;
+    c->only_bf16_theta1 = only_bf16_theta1;
     return GXPO_OK;
 }
 
@@ -859,6 +908,7 @@ gxpo_status gxpo_probe_step(gxpo_ctx* c, int which, void* stream) {
         expire_clips(c);
         return GXPO_OK;
     }
+    if (c->work_missing) return fail(c, GXPO_ERR_STATE, "this call keeps a point in `work`, which was bound as NULL");
     if (which == 0) {
         if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "probe step 0 must start a step");
         { gxpo_status fe = collect_fallback_error(c); if (fe != GXPO_OK) return fe; }
@@ -884,10 +934,25 @@ gxpo_status gxpo_probe_step(gxpo_ctx* c, int which, void* stream) {
     return GXPO_OK;
 }
 
+// theta-tilde as bfloat16 only: theta^t has to survive in `theta` and m, v have to stay put until
+// the slow step, which recomputes theta-tilde from g0 and g1 -- that is the deferred flow under
+// the gradients-persist promise, and nothing else.  Checked before the step starts.
+static gxpo_status check_only16(gxpo_ctx* c) {
+    if (!c->grads_persist || c->gslow_shares_probe)
+        return fail(c, GXPO_ERR_STATE, "GXPO_BF16_ONLY_PROBE_POINTS needs gxpo_set_gradients_persist(ctx, 1) and a g_slow buffer apart from g0 and g1: the slow step recomputes theta-tilde from them");
+    if (c->diag_on) return fail(c, GXPO_ERR_STATE, "GXPO_BF16_ONLY_PROBE_POINTS does not go with diagnostics");
+    if (c->variant == 1 || c->variant == 2)
+        return fail(c, GXPO_ERR_STATE, "GXPO_BF16_ONLY_PROBE_POINTS runs in the shared-memory staged sweeps only (gxpo_tune variant 0 or 3)");
+    return GXPO_OK;
+}
+
 gxpo_status gxpo_probe_step_deferred(gxpo_ctx* c, void* stream) {
     if (!c) return GXPO_ERR_INVALID_ARG;
     if (!c->bound) return fail(c, GXPO_ERR_STATE, "nothing bound: call gxpo_bind first");
     if (c->phase != IDLE) return fail(c, GXPO_ERR_STATE, "probe step 0 must start a step");
+    if (c->only_bf16_theta1 == 2) { gxpo_status os = check_only16(c); if (os != GXPO_OK) return os; }
+    if (c->work_missing && !c->only_bf16_theta1)
+        return fail(c, GXPO_ERR_STATE, "theta^{t,1} goes to `work`, which was bound as NULL (bind bfloat16 copies with GXPO_BF16_ONLY_THETA1 or GXPO_BF16_ONLY_PROBE_POINTS)");
     { gxpo_status fe = collect_fallback_error(c); if (fe != GXPO_OK) return fe; }
     { gxpo_status fg = finish_gate(c); if (fg != GXPO_OK) return fg; }
     if (!gate_active(c)) return fail(c, GXPO_ERR_STATE, "gate has tripped (s*=%lld, t=%lld): only fallback steps are legal", c->s_star, c->t);
@@ -896,7 +961,7 @@ gxpo_status gxpo_probe_step_deferred(gxpo_ctx* c, void* stream) {
     StepParams p = (c->cfg.placement == GXPO_PLACE_PINGPONG) ? make_step_params(c, 0, 0, 1, 0, 0)
                                                              : make_step_params(c, 0, 0, 0, 1, 0);
     p.write_state = 0;
-    p.skip_out = c->only_bf16_theta1;
+    p.skip_out = c->only_bf16_theta1 ? 1 : 0;
     gxpo_status st = launch_step(c, (cudaStream_t)stream, c->d_descs, c->d_chunks, c->num_chunks, none, p, c->d_sumsq);
     if (st != GXPO_OK) { c->t_opt -= 1; return st; }
     c->phase = PROBED0_DEFERRED;
@@ -918,9 +983,17 @@ gxpo_status gxpo_probe_extrapolate(gxpo_ctx* c, void* stream) {
     if (!c) return GXPO_ERR_INVALID_ARG;
     if (c->phase != PROBED0 && c->phase != PROBED0_DEFERRED)
         return fail(c, GXPO_ERR_STATE, "fused probe+extrapolate must follow probe step 0");
+    if (c->work_missing && c->only_bf16_theta1 != 2 && c->cfg.placement != GXPO_PLACE_PINGPONG)
+        return fail(c, GXPO_ERR_STATE, "this placement keeps theta^t in `work`, which was bound as NULL");
     const TensorDesc none = {};
     const int place = c->cfg.placement;
     const bool defer = c->phase == PROBED0_DEFERRED;
+    const bool only16 = c->only_bf16_theta1 == 2;      // theta-tilde as bfloat16 only
+    if (only16) {
+        if (!defer) return fail(c, GXPO_ERR_STATE, "GXPO_BF16_ONLY_PROBE_POINTS: take the first probe step with gxpo_probe_step_deferred");
+        gxpo_status os = check_only16(c);
+        if (os != GXPO_OK) return os;
+    }
     FusedParams p;
     p.step0 = make_step_params(c, 0, 0, 0, 0, 0);       // constants of the first probe step (replayed when deferred)
     c->t_opt += 1;
@@ -936,11 +1009,18 @@ gxpo_status gxpo_probe_extrapolate(gxpo_ctx* c, void* stream) {
     const bool lag = defer && c->grads_persist && !c->gslow_shares_probe && c->opt.kind == GXPO_OPT_ADAMW &&
                      !c->diag_on &&
                      (c->variant == 3 || (c->variant == 0 && c->num_chunks >= 8LL * c->sm_count));
-    if (lag) p.step.write_state = 0;
-    gxpo_status st = launch_fused(c, (cudaStream_t)stream, c->d_descs, c->d_chunks, c->num_chunks, none, p, defer,
-                                  c->diag_on != 0);
+    if (lag || only16) p.step.write_state = 0;
+    gxpo_status st;
+    if (only16) {
+        p.step.skip_out = 1;
+        c->lag_fused = p;
+        st = c->num_chunks > 0 ? launch_fused_bulk(c, (cudaStream_t)stream, c->d_descs, c->d_chunks, c->num_chunks, none, p, true, false)
+                               : GXPO_OK;
+    } else {
+        st = launch_fused(c, (cudaStream_t)stream, c->d_descs, c->d_chunks, c->num_chunks, none, p, defer, c->diag_on != 0);
+    }
     if (st != GXPO_OK) { c->t_opt -= 1; return st; }
-    c->state_lag = lag ? 1 : 0;
+    c->state_lag = only16 ? 2 : (lag ? 1 : 0);
     c->phase = EXTRAPOLATED;
     return GXPO_OK;
 }
@@ -953,6 +1033,13 @@ gxpo_status gxpo_slow_step(gxpo_ctx* c, void* stream) {
     StepParams p = make_step_params(c, 2, 0, 0, 0, 1);
     // diagnostics: <g0, g_slow> rides along in the staged sweep (one more read of g0);
     // otherwise it is a pass of its own over both gradients
+    if (c->state_lag == 2) {
+        gxpo_status st2 = launch_slow_recompute(c, (cudaStream_t)stream, p, c->user_sumsq ? c->user_sumsq : c->d_sumsq);
+        if (st2 != GXPO_OK) { c->t_opt -= 1; return st2; }
+        c->state_lag = 0;
+        c->phase = SLOW_DONE;
+        return GXPO_OK;
+    }
     if (c->state_lag) {
         p.replay = 1;
         p.gscale_r0 = c->gscale[0];

@@ -225,7 +225,7 @@ __device__ __forceinline__ void fused_bulk_body(const TensorDesc* __restrict__ d
                 const float x = fused_elem<ADAMW, DEFER, DIAG>(DEFER ? 0.0f : U.t1[e], U.t0[e], mm, vv,
                                                                 __fmul_rn(ld_grad1(U.g0 + e), gs0),
                                                                 __fmul_rn(ld_grad1(U.g1 + e), gs1), p, &acc);
-                U.out[e] = x;
+                if (!p.step.skip_out) U.out[e] = x;
                 if (U.wb) U.wb[e] = to_bf16(x);
                 if (ADAMW && !LIGHT && p.step.write_state) { U.m[e] = mm; U.v[e] = vv; }
             }
@@ -260,7 +260,7 @@ __device__ __forceinline__ void fused_bulk_body(const TensorDesc* __restrict__ d
             }
             optim_step_vec<ADAMW, 8>(a1, mm, vv, b1, p.step);
             extrapolate_vec<8, DIAG>(a1, a0, b0, b1, p.ex, &acc);
-            st_f(U.out + e, a1);
+            if (!p.step.skip_out) st_f(U.out + e, a1);
             if (U.wb) st_bf16(U.wb + e, a1);
             if (ADAMW && !LIGHT && p.step.write_state) { st_f(U.m + e, mm); st_f(U.v + e, vv); }
             }
@@ -554,6 +554,147 @@ step_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restric
                 *ticket = 0u;
             }
         }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// The slow step for trainers whose model runs on the bfloat16 copies only: the fused sweep
+// stored theta-tilde as bfloat16 and nothing else (theta^t is still in `theta`, m and v still
+// predate the probe steps), so this sweep stages theta^t, m, v, g_slow, g0 and g1 -- the very
+// arrays of the replaying sweep -- redoes both probe steps and the extrapolation in registers
+// with the functions of the fused sweep (hence the same float32 theta-tilde, bit for bit, whose
+// rounding the caller's third backward pass saw), and takes the slow step from there:
+// 18 R + 12 W (+2 for the bfloat16 copy of theta^{t+1}), and no float32 theta-tilde or
+// theta^{t,1} ever reaches memory.
+// ---------------------------------------------------------------------------
+// SHAPE 0: one CTA per SM, two stages of 4096 elements (the replaying sweep's ring).
+// SHAPE 1: two CTAs per SM, three stages of 2048 elements each (the light fused sweep's ring):
+// this sweep carries the arithmetic of both, and eight consumer warps per SM cannot hide it.
+template <typename G, int SHAPE>
+struct RecomputeLayout {
+    static constexpr int kMult = SHAPE ? 1 : 2;
+    static constexpr int kStagesN = SHAPE ? 3 : 2;
+    static constexpr int kElems = kTile * kMult;
+    static constexpr unsigned kF = kElems * sizeof(float);
+    static constexpr unsigned kGb = kElems * sizeof(G);
+    static constexpr unsigned kStage = 3 * kF + 3 * kGb;       // theta^t, m, v, g_slow, g0, g1
+    static constexpr unsigned kTotal = kStagesN * kStage + 2 * kMaxStages * sizeof(uint64_t) + 16;
+};
+template <typename G, int SHAPE>
+__global__ void __launch_bounds__(kBulkThreads, SHAPE ? 2 : 1)
+slow_recompute_bulk_kernel(const TensorDesc* __restrict__ descs, const ChunkRef* __restrict__ chunks,
+                           long long num_chunks, TensorDesc flat, FusedParams fp, StepParams p, int unit_shift,
+                           double* partials, unsigned* ticket, double* sumsq_out, int* error_word) {
+    typedef RecomputeLayout<G, SHAPE> L;
+    constexpr int kStages = L::kStagesN;
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ double red[8];
+    __shared__ bool is_last;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStages * L::kStage);
+    uint64_t* empty = full + kMaxStages;
+    volatile int* stop = reinterpret_cast<volatile int*>(empty + kMaxStages);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, kConsumerWarps); }
+        *stop = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const long long num_units = num_chunks << unit_shift;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (warp == kConsumerWarps) {                       // ---- producer: same stage layout as the replaying sweep
+        if (lane != 0) return;
+        unsigned it = 0; bool ok = true;
+        for (long long u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
+            StepUnit<G> U;
+            if (!step_resolve<true, G, kStepReplay>(u, unit_shift, descs, chunks, flat, p, L::kElems, U)) continue;
+            for (int j = 0; j < U.full_tiles; ++j, ++it) {
+                const unsigned s = it % kStages, n = it / kStages;
+                if (n > 0 && !mbar_wait_bounded(empty + s, (n - 1) & 1, stop, kWaitLimit)) { ok = false; break; }
+                unsigned char* st = smem + s * L::kStage;
+                const int e = j * L::kElems;
+                mbar_expect_tx(full + s, L::kStage);
+                unsigned o = 0;
+                bulk_load(st, U.in + e, L::kF, full + s); o += L::kF;
+                bulk_load(st + o, U.m + e, L::kF, full + s); o += L::kF;
+                bulk_load(st + o, U.v + e, L::kF, full + s); o += L::kF;
+                bulk_load(st + o, U.g + e, L::kGb, full + s); o += L::kGb;
+                bulk_load(st + o, U.g0 + e, L::kGb, full + s); o += L::kGb;
+                bulk_load(st + o, U.g1 + e, L::kGb, full + s);
+            }
+        }
+        if (!ok) {
+            *stop = 1; atomicExch(error_word, 1);
+            for (unsigned k = 0; k < (unsigned)kStages && k < it; ++k) {
+                const unsigned i2 = it - 1 - k;
+                for (unsigned w = 0; w < kWaitLimit && !mbar_try_wait(full + i2 % kStages, (i2 / kStages) & 1); ++w) __nanosleep(64);
+            }
+        }
+        return;
+    }
+    const float gscale = p.gscale ? __ldg(p.gscale) : 1.0f;
+    const float gs0 = fp.ex.gscale0 ? __ldg(fp.ex.gscale0) : 1.0f, gs1 = fp.ex.gscale1 ? __ldg(fp.ex.gscale1) : 1.0f;
+    double acc = 0.0; unsigned it = 0; bool alive = true;
+    for (long long u = blockIdx.x; u < num_units && alive; u += gridDim.x) {
+        StepUnit<G> U;
+        if (!step_resolve<true, G, kStepReplay>(u, unit_shift, descs, chunks, flat, p, L::kElems, U)) continue;
+        for (int j = 0; j < U.full_tiles; ++j, ++it) {
+            const unsigned s = it % kStages, n = it / kStages;
+            if (!mbar_wait_bounded(full + s, n & 1, stop, kWaitLimit)) { *stop = 1; atomicExch(error_word, 1); alive = false; break; }
+            const unsigned char* st = smem + s * L::kStage;
+#pragma unroll 1
+            for (int h = 0; h < L::kMult; ++h) {
+                const int tt = (h * kThreads + threadIdx.x) * 8;
+                unsigned o = 0;
+                const FVec<8> th0 = lds_f8(reinterpret_cast<const float*>(st) + tt); o += L::kF;
+                FVec<8> mm = lds_f8(reinterpret_cast<const float*>(st + o) + tt); o += L::kF;
+                FVec<8> vv = lds_f8(reinterpret_cast<const float*>(st + o) + tt); o += L::kF;
+                const FVec<8> gg = lds_g8(reinterpret_cast<const G*>(st + o) + tt); o += L::kGb;
+                const FVec<8> b0 = scaled<8>(lds_g8(reinterpret_cast<const G*>(st + o) + tt), gs0); o += L::kGb;
+                const FVec<8> b1 = scaled<8>(lds_g8(reinterpret_cast<const G*>(st + o) + tt), gs1);
+                FVec<8> th = th0;
+                optim_step_vec<true, 8>(th, mm, vv, b0, fp.step0);
+                optim_step_vec<true, 8>(th, mm, vv, b1, fp.step);
+                extrapolate_vec<8, false>(th, th0, b0, b1, fp.ex, nullptr);          // th = theta-tilde
+                float sq = 0.0f;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) sq = fmaf(gg.x[i], gg.x[i], sq);
+                optim_step_vec<true, 8>(th, mm, vv, scaled<8>(gg, gscale), p);      // same roundings as optim_step_elem
+                const int e = j * L::kElems + tt;
+                st_f(U.out + e, th);
+                if (U.wb) st_bf16(U.wb + e, th);
+                st_f(U.m + e, mm); st_f(U.v + e, vv);
+                acc += (double)sq;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty + s);
+        }
+        if (!alive) break;
+        // what bypasses the ring (ragged ends, misaligned tensors): coordinate by coordinate
+        for (int e = U.full_tiles * L::kElems + threadIdx.x; e < U.len; e += kThreads) {
+            float mm = U.m[e], vv = U.v[e];
+            const float gg = ld_grad1(U.g + e);
+            float x = fused_elem<true, true, false>(0.0f, U.in[e], mm, vv, __fmul_rn(ld_grad1(U.g0 + e), gs0),
+                                                    __fmul_rn(ld_grad1(U.g1 + e), gs1), fp, nullptr);
+            optim_step_elem<true>(x, mm, vv, __fmul_rn(gg, gscale), p);
+            U.out[e] = x;
+            if (U.wb) U.wb[e] = to_bf16(x);
+            U.m[e] = mm; U.v[e] = vv;
+            acc += (double)(gg * gg);
+        }
+    }
+    const double tot = consumer_sum(acc, red);
+    if (threadIdx.x == 0) {
+        partials[blockIdx.x] = tot;
+        __threadfence();
+        is_last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+    }
+    asm volatile("bar.sync 1, %0;" :: "r"(kThreads) : "memory");
+    if (is_last) {
+        __threadfence();
+        double sum = 0.0;
+        for (unsigned i = threadIdx.x; i < gridDim.x; i += kThreads) sum += __ldcg(partials + i);
+        sum = consumer_sum(sum, red);
+        if (threadIdx.x == 0) { *sumsq_out = sum; *ticket = 0u; }
     }
 }
 

@@ -111,7 +111,8 @@ def _one_active_step_vs_oracle(workload, lr, picks_fn, full_oracle_norm, extra_w
         for _, k in shapes:
             offs.append(acc)
             acc += k
-        ctx.bind_model_weights([weights.data_ptr() + 2 * o for o in offs], only_bf16_theta1=True)
+        ctx.bind_model_weights([weights.data_ptr() + 2 * o for o in offs],
+                               bf16_only=b.BF16_ONLY_THETA1 if alias else emit)
     gcfg, ocfg = gu.ora_cfgs(cfg, opt)
     wins = _windows(shapes, picks_fn(shapes)) + list(extra_windows)
     before = [_grab(keep, lo, hi) for lo, hi in wins]
@@ -172,11 +173,14 @@ def test_flat_1p54b_other_depths(K):
     _one_active_step_vs_oracle("flat_1p54b", 1e-3, picks, full_oracle_norm=False, K=K)
 
 
-def test_flat_1p54b_with_bf16_model_weight_copies():
-    """bench.py --emit-bf16 at full size: same float32 results, and the bfloat16 copies."""
+@pytest.mark.parametrize("mode", [1, 2])
+def test_flat_1p54b_with_bf16_model_weight_copies(mode):
+    """bench.py --emit-bf16 at full size: same float32 results, and the bfloat16 copies.
+    mode 1: theta^{t,1} as bfloat16 only; mode 2 (the benchmark's): theta-tilde too, recomputed
+    by the slow step."""
     def picks(shapes):
         return [(0, "head"), (0, "chunk"), (0, "tail")]
-    _one_active_step_vs_oracle("flat_1p54b", 1e-3, picks, full_oracle_norm=False, emit=True)
+    _one_active_step_vs_oracle("flat_1p54b", 1e-3, picks, full_oracle_norm=False, emit=mode)
 
 
 def test_flat_2p5b_offsets_beyond_two_to_the_31():

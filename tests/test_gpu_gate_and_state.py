@@ -167,14 +167,19 @@ def test_call_order_and_argument_checks():
     pr = gu.Problem(th, m, v, g0, g1, gs)
     good = pr.ptrs()
     for field, val, status in [("n", -1, b.ERR_INVALID_ARG), ("theta", 0, b.ERR_INVALID_ARG),
-                               ("work", 0, b.ERR_INVALID_ARG), ("m", 0, b.ERR_INVALID_ARG),
-                               ("g_slow", 0, b.ERR_INVALID_ARG),
+                               ("m", 0, b.ERR_INVALID_ARG), ("g_slow", 0, b.ERR_INVALID_ARG),
                                ("theta", good.theta + 2, b.ERR_ALIGNMENT),
                                ("g1", good.g1 + 1, b.ERR_ALIGNMENT)]:
         t = b.TensorPtrs(**{**good.__dict__, field: val})
         with pytest.raises(b.GxpoError) as e:
             ctx.bind([t])
         assert e.value.status == status, field
+    # `work` may be left out at bind time; the calls that keep a point there then refuse
+    ctx.bind([b.TensorPtrs(**{**good.__dict__, "work": 0})])
+    for call in (lambda: ctx.probe_step(0), ctx.probe_step_deferred):
+        with pytest.raises(b.GxpoError) as e:
+            call()
+        assert e.value.status == b.ERR_STATE and "work" in str(e.value)
     ctx.bind([good])
     for call in (lambda: ctx.probe_step(1), ctx.extrapolate, ctx.slow_step, ctx.gate_update):
         with pytest.raises(b.GxpoError) as e:

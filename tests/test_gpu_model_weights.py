@@ -156,3 +156,131 @@ def test_binding_rules():
     for w, x in zip(wbs, before):
         np.testing.assert_array_equal(_bits(w), x)
     ctx.close()
+
+
+@pytest.mark.parametrize("variant", [0, 3])
+@pytest.mark.parametrize("bind_work", [True, False])
+def test_bf16_only_probe_points_is_bit_identical_and_never_touches_work(variant, bind_work):
+    """GXPO_BF16_ONLY_PROBE_POINTS: theta^{t,1} and theta-tilde exist as bfloat16 copies only,
+    theta^t stays in `theta` and m, v stay put until the slow step, which recomputes
+    theta-tilde.  Over three steps every copy and every float32 result must equal, bit for
+    bit, what the same steps give with all float32 points stored (a flow the oracle checks
+    above); `work` may be bound as NULL."""
+    import torch
+    b = _binding()
+    a_p, a_ctx, cfg, opt, a_w = _setup(b, "adamw", 0, True)                     # float32 points beside the copies
+    b_p, b_ctx, _, _, b_w = _setup(b, "adamw", 0, False)
+    if not bind_work:
+        b_ctx.bind([b.tensor_ptrs(p.theta, None, p.m, p.v, p.g0, p.g1, p.gs) for p in b_p])
+    b_w = []
+    for p, off in zip(b_p, OFFSETS):
+        big = torch.full((p.n + off + 16,), float("nan"), dtype=torch.bfloat16, device="cuda")
+        b_w.append(big[off:off + p.n])
+        p.work.fill_(123.0)
+    b_ctx.bind_model_weights([w.data_ptr() for w in b_w], bf16_only=b.BF16_ONLY_PROBE_POINTS)
+    for c in (a_ctx, b_ctx):
+        c.tune(0, variant, 0)
+        c.set_gradients_persist(True)
+    for step in range(3):
+        start = [(gu.to_host_f64(p.theta), gu.to_host_f64(p.m), gu.to_host_f64(p.v)) for p in b_p]
+        a_ctx.probe_step_deferred(); b_ctx.probe_step_deferred()
+        for wa, wb in zip(a_w, b_w):
+            np.testing.assert_array_equal(_bits(wa), _bits(wb), err_msg=f"step {step}: theta1 copy")
+        a_ctx.probe_extrapolate(); b_ctx.probe_extrapolate()
+        k = b_ctx.last_sweep()
+        assert (k.kernel, k.bytes_read_per_param, k.bytes_written_per_param) == (b"fused_bulk_light_kernel", 16, 2)
+        for p, wa, wb, s0 in zip(b_p, a_w, b_w, start):
+            np.testing.assert_array_equal(_bits(wa), _bits(wb), err_msg=f"step {step}: theta-tilde copy")
+            np.testing.assert_array_equal(gu.to_host_f64(p.theta), s0[0])      # theta^t still in place
+            np.testing.assert_array_equal(gu.to_host_f64(p.m), s0[1])          # m, v still unwritten
+            np.testing.assert_array_equal(gu.to_host_f64(p.v), s0[2])
+        a_ctx.slow_step(); b_ctx.slow_step()
+        k = b_ctx.last_sweep()
+        assert (k.kernel, k.bytes_read_per_param, k.bytes_written_per_param) == (b"slow_recompute_bulk_kernel", 18, 14)
+        ra, rb = a_ctx.gate_update(allow_nonfinite=True), b_ctx.gate_update(allow_nonfinite=True)
+        for i, (p, q, wa, wb) in enumerate(zip(a_p, b_p, a_w, b_w)):
+            for nm in ("theta", "m", "v"):
+                np.testing.assert_array_equal(gu.to_host_f64(getattr(p, nm)), gu.to_host_f64(getattr(q, nm)),
+                                              err_msg=f"step {step}, tensor {i}: {nm}")
+            np.testing.assert_array_equal(_bits(wa), _bits(wb), err_msg=f"step {step}: theta^{{t+1}} copy")
+            assert torch.all(q.work == 123.0)                                  # never written
+        # the norm's float32 partial sums are grouped by the sweep's shape (tiles of 8 here, single
+        # coordinates in the ragged ends there): equal to float32 rounding of the groups, not to the bit
+        assert rb.norm == pytest.approx(ra.norm, rel=1e-7)
+    assert a_ctx.launch_count() == b_ctx.launch_count() == 12
+    # the fallback step needs no `work` either and emits its copy
+    b_ctx.probe_step(-1)
+    for p, w in zip(b_p, b_w):
+        _assert_copy_of(w, p.theta, "fallback copy")
+    a_ctx.close(); b_ctx.close()
+
+
+def test_bf16_only_probe_points_against_the_oracle():
+    b = _binding()
+    probs, ctx, cfg, opt, wbs = _setup(b, "adamw", 0, True)
+    ctx.bind_model_weights([w.data_ptr() for w in wbs], bf16_only=b.BF16_ONLY_PROBE_POINTS)
+    ctx.set_gradients_persist(True)
+    gcfg, ocfg = gu.ora_cfgs(cfg, opt)
+    res = ctx.active_step(allow_nonfinite=True, deferred=True)
+    sumsq = 0.0
+    for i, (p, w) in enumerate(zip(probs, wbs)):
+        st = p.oracle_state(ocfg)
+        grads = p.oracle_grads()
+        tr = {}
+        ora.active_step(st, gcfg, lambda k, th: grads[k], round_f32=True, trace=tr)
+        sat = ~np.isfinite(tr["scale"]) | (np.abs(tr["scale"]) > 1e30)
+        slack = gu.displacement_slack(p.np_in["theta"].astype(np.float64), tr["theta2"], tr["scale"], gcfg.alpha,
+                                      theta1=tr["theta1"])
+        gu.assert_close(gu.to_host_f64(p.theta), st.theta, f"tensor {i} theta", rtol=2e-6, saturated=sat, extra_abs=slack)
+        gu.assert_close(gu.to_host_f64(p.m), st.m, f"tensor {i} m")
+        gu.assert_close(gu.to_host_f64(p.v), st.v, f"tensor {i} v")
+        _assert_copy_of(w, p.theta, "theta^{t+1} copy")
+        sumsq += ora.sum_squares(grads[2])
+    assert res.norm == pytest.approx(np.sqrt(sumsq), rel=gu.RTOL_NORM)
+    ctx.close()
+
+
+def test_bf16_only_probe_points_rules():
+    b = _binding()
+    probs, ctx, cfg, opt, wbs = _setup(b, "adamw", 0, True)
+    ptrs = [w.data_ptr() for w in wbs]
+    ctx.bind_model_weights(ptrs, bf16_only=b.BF16_ONLY_PROBE_POINTS)
+    with pytest.raises(b.GxpoError) as e:                     # no promise: refused before the step starts
+        ctx.probe_step_deferred()
+    assert e.value.status == b.ERR_STATE and "gradients_persist" in str(e.value)
+    ctx.set_gradients_persist(True)
+    ctx.probe_step(0)                                         # the non-deferred first step is legal ...
+    with pytest.raises(b.GxpoError) as e:
+        ctx.probe_extrapolate()                               # ... but this mode cannot follow it
+    assert e.value.status == b.ERR_STATE
+    ctx.probe_step(1); ctx.extrapolate(); ctx.slow_step(); ctx.gate_update(allow_nonfinite=True)
+    ctx.enable_diagnostics(True)
+    with pytest.raises(b.GxpoError) as e:
+        ctx.probe_step_deferred()
+    assert e.value.status == b.ERR_STATE and "diagnostics" in str(e.value)
+    ctx.enable_diagnostics(False)
+    ctx.tune(0, 2, 0)
+    with pytest.raises(b.GxpoError) as e:
+        ctx.probe_step_deferred()
+    assert e.value.status == b.ERR_STATE
+    ctx.tune(0, 0, 0)
+    assert ctx.active_step(allow_nonfinite=True, deferred=True).t == 2
+    with pytest.raises(b.GxpoError) as e:
+        ctx.bind_model_weights(ptrs, bf16_only=3)
+    assert e.value.status == b.ERR_INVALID_ARG
+    ctx.close()
+    # work == NULL: only the calls that keep no point there
+    ctx = b.Context(cfg, opt, b.BF16)
+    ctx.bind([b.tensor_ptrs(p.theta, None, p.m, p.v, p.g0, p.g1, p.gs) for p in probs])
+    for call in (lambda: ctx.probe_step(0), lambda: ctx.probe_step_deferred()):
+        with pytest.raises(b.GxpoError) as e:
+            call()
+        assert e.value.status == b.ERR_STATE and "work" in str(e.value)
+    ctx.probe_step(-1)                                        # the fallback step works in place
+    ctx.close()
+    # plain gradient descent: not built
+    gp, gctx, _, _, gw = _setup(b, "gd", 0, True)
+    with pytest.raises(b.GxpoError) as e:
+        gctx.bind_model_weights([w.data_ptr() for w in gw], bf16_only=b.BF16_ONLY_PROBE_POINTS)
+    assert e.value.status == b.ERR_INVALID_ARG
+    gctx.close()
