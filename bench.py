@@ -393,7 +393,9 @@ def run_ours(args):
     G = 2                                                     # bfloat16 gradients
     relabel = {}
     if "probe_extrapolate_deferred" in sweeps and sweeps["probe_extrapolate_deferred"].kernel == b"fused_bulk_light_kernel":
-        relabel["probe_extrapolate_deferred"] = "probe_extrapolate_nostate"      # m, v left unwritten
+        relabel["probe_extrapolate_deferred"] = ("probe_extrapolate_nostate"     # m, v left unwritten
+                                                 if sweeps["probe_extrapolate_deferred"].bytes_written_per_param >= 4 else
+                                                 "probe_extrapolate_bf16only")   # and theta-tilde as bfloat16 only
     if "slow_step" in sweeps and sweeps["slow_step"].kernel == b"slow_recompute_bulk_kernel":
         relabel["slow_step"] = "slow_step_recompute"                             # theta-tilde redone from theta^t, g0, g1
     elif "slow_step" in sweeps and sweeps["slow_step"].bytes_read_per_param - sweeps["slow_step"].extra_launches * 2 * G == 12 + 3 * G:
@@ -467,7 +469,9 @@ def run_ours(args):
                    "K": args.K, "alpha": args.alpha, "lr": args.lr, "grad_dtype": "bf16",
                    "placement": ["pingpong", "snapshot"][args.placement],
                    "step": "fallback (single pass)" if args.fallback else
-                   {"deferred": ("active (probe with deferred state, probe+extrapolate in one sweep with m, v still unwritten, "
+                   {"deferred": ("active (probe with deferred state writing bfloat16 theta1 only, probe+extrapolate in one sweep "
+                                 "writing bfloat16 theta-tilde only, slow step recomputing theta-tilde, gate)") if only16 else
+                                ("active (probe with deferred state, probe+extrapolate in one sweep with m, v still unwritten, "
                                  "slow step replaying both moment updates, gate)") if lag else
                                 "active (probe with deferred state, probe+extrapolate in one sweep, slow step, gate)",
                     "fused": "active (probe, probe+extrapolate in one sweep, slow step, gate)",

@@ -7,6 +7,9 @@ The check: through the C ABI, on the same theta-tilde, m, v and g_slow, it must 
 what gxpo_slow_step + gxpo_gate_update give -- parameters and optimizer state within
 the element tolerance of the parity tests, the norm within the norm tolerance -- on two
 calls in a row (the second call reuses the scratch the first one left behind).
+Further cases hold it against the CPU oracle directly: a buffer with more chunks than the
+grid has CTAs, a short buffer right after it, a single parameter, and two calls on two
+streams ordered by an event.
 
 This file is named so that pytest collects it last; it depends on nothing the other
 tests do and passes in a fresh process as well."""
