@@ -214,6 +214,18 @@ int unit_shift_for(const gxpo_ctx* c, long long num_chunks) {
     return sh;
 }
 
+// (x, x) as one 64-bit word, for the two-lane instructions
+unsigned long long pair_of(float x) {
+    unsigned u;
+    std::memcpy(&u, &x, sizeof(u));
+    return ((unsigned long long)u << 32) | u;
+}
+void fill_step_pairs(StepParams& p) {
+    p.beta1_2 = pair_of(p.beta1); p.beta2_2 = pair_of(p.beta2); p.omb1_2 = pair_of(p.omb1); p.omb2_2 = pair_of(p.omb2);
+    p.eps_2 = pair_of(p.eps); p.inv_sqrt_bc2_2 = pair_of(p.inv_sqrt_bc2); p.step_2 = pair_of(p.step_size);
+    p.decay_2 = pair_of(p.decay); p.neg_lr_2 = pair_of(-p.lr);
+}
+
 StepParams make_step_params(gxpo_ctx* c, int which_grad, int in_sel, int out_sel, int snapshot,
                             int want_norm) {
     StepParams p;
@@ -241,6 +253,7 @@ StepParams make_step_params(gxpo_ctx* c, int which_grad, int in_sel, int out_sel
         p.step_size = (float)(lr / (1.0 - std::pow(b1, t)));
         p.inv_sqrt_bc2 = (float)(1.0 / std::sqrt(1.0 - std::pow(b2, t)));
     }
+    fill_step_pairs(p);
     return p;
 }
 
@@ -525,6 +538,7 @@ ExtrapParams make_extrap_params(const gxpo_ctx* c, int placement) {
     p.alpha = c->cfg.alpha;
     p.delta = c->cfg.delta;
     p.den_eps = c->cfg.den_eps;
+    p.alpha_2 = pair_of(p.alpha); p.one_2 = pair_of(1.0f); p.neg_one_2 = pair_of(-1.0f);
     p.gscale0 = c->gscale[0];
     p.gscale1 = c->gscale[1];
     if (placement == GXPO_PLACE_PINGPONG) { p.theta2_sel = 1; p.theta0_sel = 0; }
@@ -1615,6 +1629,7 @@ extern "C" gxpo_status gxpo_slow_step_noalloc(float* theta, float* m, float* v, 
         p.step_size = (float)(lr / (1.0 - std::pow(b1, t)));
         p.inv_sqrt_bc2 = (float)(1.0 / std::sqrt(1.0 - std::pow(b2, t)));
     }
+    fill_step_pairs(p);
     TensorDesc d;
     std::memset(&d, 0, sizeof(d));
     d.theta = theta; d.m = m; d.v = v; d.g[2] = g_slow; d.n = n;
