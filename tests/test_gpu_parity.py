@@ -247,6 +247,27 @@ def test_access_variants_and_launch_shapes_agree_bitwise():
         assert o[3] == pytest.approx(outs[0][3], rel=1e-7)
 
 
+def test_run_to_run_determinism_with_bf16_only_probe_points():
+    """The recomputing slow sweep sums sum(g_slow^2) in a fixed order as well."""
+    import torch
+    b = _binding()
+    n = 5 * 32768 + 4096 + 11
+    got = []
+    for _ in range(2):
+        pr = _problem(n, seed=5, grad_dtype="bf16")
+        ctx, cfg, opt = _ctx(b, "bf16", lr=1e-3)
+        ctx.bind([pr.ptrs()])
+        wb = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
+        ctx.bind_model_weights([wb.data_ptr()], bf16_only=b.BF16_ONLY_PROBE_POINTS)
+        ctx.set_gradients_persist(True)
+        res = [ctx.active_step(allow_nonfinite=True, deferred=True).norm for _ in range(2)]
+        got.append((gu.to_host_f64(pr.theta), gu.to_host_f64(pr.m), gu.to_host_f64(wb), res))
+        ctx.close()
+    for x, y in zip(got[0][:3], got[1][:3]):
+        np.testing.assert_array_equal(x, y)
+    assert got[0][3] == got[1][3]
+
+
 @pytest.mark.parametrize("staged", [False, True])
 def test_run_to_run_determinism(staged):
     """Two runs on the same bits give the same bits, the norm included: the reductions have a
@@ -417,16 +438,21 @@ def test_fused_call_order():
 
 
 @pytest.mark.parametrize("flow,staging", [(f, s) for f in ("deferred", "fused", "unfused", "fallback")
-                                          for s in ("registers", "staged")] + [("deferred", "staged+promise")])
+                                          for s in ("registers", "staged")] + [("deferred", "staged+promise"),
+                                                                               ("deferred", "bf16-only points")])
 @pytest.mark.parametrize("placement", [0, 1])
 def test_no_sweep_writes_outside_its_tensors(flow, placement, staging):
     """Every output buffer (theta, work, m, v and the bfloat16 copies) sits between two
     guard bands filled with a sentinel; after a step the bands must be untouched and the
     read-only gradient buffers bit-identical.  Sizes end mid-vector, mid-tile, mid-stage and
     mid-chunk, aligned and misaligned; the shared-memory staged sweeps (with and without the
-    gradients-persist promise, which needs diagnostics off) are held to the same."""
+    gradients-persist promise, which needs diagnostics off) are held to the same, and so is
+    the step with bfloat16-only probe points, which must not touch `work` at all."""
     import torch
     b = _binding()
+    only16 = staging == "bf16-only points"
+    if only16 and placement == 1:
+        pytest.skip("bfloat16-only points need PINGPONG placement")
     sizes = [1, 7, 2049, 32768 + 3, 2 * 32768 - 1, 70001, 3 * 4096 + 2048 + 5]
     offsets = [0, 3, 0, 0, 1, 0, 0]
     GUARD = 4096
@@ -452,10 +478,11 @@ def test_no_sweep_writes_outside_its_tensors(flow, placement, staging):
         grads.append((pr, [pr.g0.clone(), pr.g1.clone(), pr.gs.clone()]))
     ctx, cfg, opt = _ctx(b, "bf16", lr=1e-3, K=5, alpha=0.5, placement=placement)
     ctx.bind(ptrs)
-    ctx.bind_model_weights(wptrs)
+    ctx.bind_model_weights(wptrs, bf16_only=b.BF16_ONLY_PROBE_POINTS if only16 else b.BF16_BESIDE)
     ctx.tune(0, 2 if staging == "registers" else 3, 0)
-    ctx.enable_diagnostics(staging != "staged+promise")
-    ctx.set_gradients_persist(staging == "staged+promise")
+    ctx.enable_diagnostics(staging not in ("staged+promise", "bf16-only points"))
+    ctx.set_gradients_persist(staging in ("staged+promise", "bf16-only points"))
+    work_before = [bigs[5 * i + 1].clone() for i in range(len(sizes))] if only16 else None
     for _ in range(2):
         if flow == "fallback":
             ctx.probe_step(-1)
@@ -465,6 +492,9 @@ def test_no_sweep_writes_outside_its_tensors(flow, placement, staging):
     for big in bigs:
         s = torch.tensor(sentinel, dtype=big.dtype, device="cuda")
         assert torch.all(big[:GUARD] == s) and torch.all(big[-GUARD:] == s)
+    if only16:
+        for i, w in enumerate(work_before):
+            assert torch.equal(bigs[5 * i + 1].view(torch.int32), w.view(torch.int32)), f"tensor {i}: `work` was written"
     for pr, (g0, g1, gs) in grads:
         assert torch.equal(pr.g0.view(torch.int16), g0.view(torch.int16))
         assert torch.equal(pr.g1.view(torch.int16), g1.view(torch.int16))
