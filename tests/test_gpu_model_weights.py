@@ -284,3 +284,35 @@ def test_bf16_only_probe_points_rules():
         gctx.bind_model_weights([w.data_ptr() for w in gw], bf16_only=b.BF16_ONLY_PROBE_POINTS)
     assert e.value.status == b.ERR_INVALID_ARG
     gctx.close()
+
+
+def test_bf16_only_probe_points_with_gradient_scales_and_clipping():
+    """The recomputing slow sweep scales g0, g1 and g_slow as the sweeps before it did: a caller's
+    scale on g1 and clipping coefficients on g0 and g_slow give the same bits as with every
+    float32 point stored."""
+    import torch
+    b = _binding()
+    outs = []
+    for mode in (b.BF16_BESIDE, b.BF16_ONLY_PROBE_POINTS):
+        probs, ctx, cfg, opt, wbs = _setup(b, "adamw", 0, True)
+        ctx.bind_model_weights([w.data_ptr() for w in wbs], bf16_only=mode)
+        ctx.tune(0, 3, 0)
+        ctx.set_gradients_persist(True)
+        scale = torch.tensor([0.7], dtype=torch.float32, device="cuda")
+        ctx.set_grad_scale(1, scale.data_ptr())
+        for _ in range(2):
+            ctx.clip_grad_norm(0, 0.05)
+            ctx.probe_step_deferred()
+            ctx.probe_extrapolate()
+            ctx.clip_grad_norm(2, 0.05)
+            ctx.slow_step()
+            res = ctx.gate_update(allow_nonfinite=True)
+        outs.append(([(gu.to_host_f64(p.theta), gu.to_host_f64(p.m), gu.to_host_f64(p.v)) for p in probs],
+                     [_bits(w) for w in wbs], res.norm))
+        ctx.close()
+    for x, y in zip(outs[0][0], outs[1][0]):
+        for u, w in zip(x, y):
+            np.testing.assert_array_equal(u, w)
+    for x, y in zip(outs[0][1], outs[1][1]):
+        np.testing.assert_array_equal(x, y)
+    assert outs[1][2] == pytest.approx(outs[0][2], rel=1e-7)
