@@ -144,7 +144,7 @@ void gxpo_destroy(gxpo_ctx* ctx);
 /* Bind a tensor list (count == 1 is the flat-buffer case).  Copies the descriptors
  * and builds the chunk table on the device; the list itself is not kept.  May be
  * called again between steps to re-bind.  Before it overwrites an earlier table it waits
- * for this context's own outstanding work (the last gate read-back, the last fallback
+ * for this context's own outstanding work (the last gate update, the last fallback
  * sweep) and for nothing else: other streams of the process keep running, and no device
  * memory is freed or allocated unless the new list needs a larger table than any before.
  * Errors: INVALID_ARG (null list entry fields, n < 0, count < 0, m/v missing for
@@ -248,17 +248,18 @@ gxpo_status gxpo_slow_step(gxpo_ctx* ctx, void* stream);
 /* Adaptive rule (Eq. (z_score); Algorithm 1 after the slow correction), evaluated
  * by a device kernel: ||g_slow||, mu and sigma of the stored norms, Z, Z >= tau =>
  * s_star = t + 1; the norm is pushed either way; t advances.  Waits for `stream`
- * (one 64-byte read-back).  `out` may be NULL.  state: SLOW_DONE -> IDLE.
+ * (the kernel writes its 72-byte record straight into pinned host memory, which the host
+ * polls: no copy and no event in between).  `out` may be NULL.  state: SLOW_DONE -> IDLE.
  * Returns NONFINITE (after completing the update and tripping the gate) when the
  * norm is Inf/NaN -- that rule is this library's, not the paper's. */
 gxpo_status gxpo_gate_update(gxpo_ctx* ctx, void* stream, gxpo_gate_result* out);
 
-/* The same update without the wait: the gate kernel and its 64-byte read-back are only
+/* The same update without the wait: the gate kernel (which delivers its record itself) is only
  * enqueued on `stream`, and the call returns at once, so the host can go on issuing work
  * (the next rollouts, the next backward pass) while the step drains.  The outcome is
  * collected by whichever call needs it first: gxpo_gate_last, gxpo_gate_peek, the next
  * gxpo_probe_step(ctx, 0) / gxpo_probe_step_deferred (they must know whether the gate
- * has tripped), gxpo_backward_passes, gxpo_state_export -- each waits for the read-back
+ * has tripped), gxpo_backward_passes, gxpo_state_export -- each waits for the record
  * if it is still in flight.  state: SLOW_DONE -> IDLE. */
 gxpo_status gxpo_gate_update_async(gxpo_ctx* ctx, void* stream);
 
@@ -336,7 +337,7 @@ gxpo_status gxpo_enable_diagnostics(gxpo_ctx* ctx, int on);
 gxpo_status gxpo_get_diagnostics(gxpo_ctx* ctx, void* stream, gxpo_diagnostics* out);
 
 /* Host-side view of the gate; no device work (it only waits if a gxpo_gate_update_async
- * read-back is still in flight). */
+ * record has not arrived yet). */
 gxpo_status gxpo_gate_peek(const gxpo_ctx* ctx, int* active, long long* s_star, long long* t);
 
 /* Optimizer step count so far (3 per active step, 1 per fallback step). */

@@ -8,6 +8,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <atomic>
 #include <mutex>
 #include <new>
 #include <vector>
@@ -70,10 +71,11 @@ struct gxpo_ctx {
     double* user_sumsq;                // caller-owned replacement for d_sumsq, or null
     GateState* d_gate;
     double* d_ring;
-    GateResult* d_result;
-    GateResult* h_result;              // pinned
-    cudaEvent_t gate_done;             // recorded after the gate's read-back
-    int gate_pending;                  // a read-back is in flight (gxpo_gate_update_async)
+    GateResult* h_result;              // pinned and mapped: the gate kernel writes it directly
+    GateResult* h_result_dev;          // the same memory as the device addresses it
+    unsigned long long gate_seq;       // sequence number of the last gate update launched
+    cudaEvent_t gate_done;             // recorded after the gate kernel
+    int gate_pending;                  // a gate update is in flight (gxpo_gate_update_async)
     int have_gate;
     gxpo_gate_result last_gate;
     // per-step diagnostics (off by default)
@@ -556,11 +558,11 @@ void expire_clips(gxpo_ctx* c) {
 // Enqueue the gate kernel and its read-back; the host learns the outcome in finish_gate.
 // t advances by one whatever the outcome, so the host mirror moves on at once.
 gxpo_status launch_gate(gxpo_ctx* c, cudaStream_t s, const double* sumsq) {
+    c->gate_seq += 1;
     gate_kernel<<<1, 32, 0, s>>>(c->d_gate, c->d_ring, sumsq, c->t, c->cfg.tau, c->cfg.gate_eps,
-                                 c->cfg.window, c->cfg.min_history, c->cfg.std_ddof, c->d_err, c->d_result);
+                                 c->cfg.window, c->cfg.min_history, c->cfg.std_ddof, c->d_err, c->h_result_dev, c->gate_seq);
     c->launches += 1;
     CUDA_TRY(c, cudaGetLastError());
-    CUDA_TRY(c, cudaMemcpyAsync(c->h_result, c->d_result, sizeof(GateResult), cudaMemcpyDeviceToHost, s));
     CUDA_TRY(c, cudaEventRecord(c->gate_done, s));
     c->gate_pending = 1;
     c->t += 1;
@@ -570,7 +572,21 @@ gxpo_status launch_gate(gxpo_ctx* c, cudaStream_t s, const double* sumsq) {
 // Wait for a pending gate read-back (if any) and fold it into the host mirror.
 gxpo_status finish_gate(gxpo_ctx* c) {
     if (!c->gate_pending) return GXPO_OK;
-    CUDA_TRY(c, cudaEventSynchronize(c->gate_done));
+    // Poll the record's sequence number in host memory (the kernel writes it last); after a
+    // bounded number of polls fall back to waiting on the event, which also surfaces a failed launch.
+    volatile unsigned long long* seq = &c->h_result->seq;
+    bool seen = false;
+    for (int spin = 0; spin < (1 << 22); ++spin) {
+        if (*seq == c->gate_seq) { seen = true; break; }
+#if defined(__x86_64__) || defined(__i386__)
+        __builtin_ia32_pause();
+#endif
+    }
+    if (!seen) {
+        CUDA_TRY(c, cudaEventSynchronize(c->gate_done));
+        if (*seq != c->gate_seq) return fail(c, GXPO_ERR_CUDA, "the gate kernel finished without delivering its result");
+    }
+    std::atomic_thread_fence(std::memory_order_acquire);
     c->gate_pending = 0;
     const GateResult r = *c->h_result;
     c->s_star = r.s_star;
@@ -726,8 +742,9 @@ gxpo_status gxpo_create(const gxpo_cfg* cfg, const gxpo_opt_cfg* opt, int grad_d
     if (e == cudaSuccess) e = cudaMemset(c->d_err, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaMalloc(&c->d_gate, sizeof(GateState));
     if (e == cudaSuccess) e = cudaMalloc(&c->d_ring, (size_t)cfg->window * sizeof(double));
-    if (e == cudaSuccess) e = cudaMalloc(&c->d_result, sizeof(GateResult));
-    if (e == cudaSuccess) e = cudaMallocHost(&c->h_result, sizeof(GateResult));
+    if (e == cudaSuccess) e = cudaHostAlloc(&c->h_result, sizeof(GateResult), cudaHostAllocMapped);
+    if (e == cudaSuccess) std::memset(c->h_result, 0, sizeof(GateResult));
+    if (e == cudaSuccess) e = cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->h_result_dev), c->h_result, 0);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->gate_done, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->idle_event, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->err_done, cudaEventDisableTiming);
@@ -768,7 +785,6 @@ void gxpo_destroy(gxpo_ctx* c) {
     cudaFree(c->d_err);
     cudaFree(c->d_gate);
     cudaFree(c->d_ring);
-    cudaFree(c->d_result);
     if (c->h_result) cudaFreeHost(c->h_result);
     if (c->gate_done) cudaEventDestroy(c->gate_done);
     if (c->idle_event) cudaEventDestroy(c->idle_event);
