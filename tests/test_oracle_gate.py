@@ -176,3 +176,24 @@ def test_outer_loop_counts_backward_passes(row):
     assert gate.s_star == s_star
     assert calls["n"] == passes == total
     assert st.t_opt == total                              # one optimizer step per backward pass
+
+
+def test_z_score_is_invariant_to_shift_and_positive_scale_of_the_norm_stream():
+    """Z = (x - mu) / (sigma + eps) (Eq. (z_score)): adding a constant to every norm changes
+    nothing, and with eps = 0 neither does multiplying them by c > 0 -- so the gate flips at the
+    same step.  A mean taken over the wrong window, a variance without the mean removed or a
+    sigma that is a variance all break one of the two."""
+    t = np.arange(60)
+    norms = 1.0 + 0.05 * (-1.0) ** t + 0.01 * np.sin(t)       # |Z| stays near 1 from the second entry on
+    norms[37] += 0.5                                          # a clear upward jump: Z ~ 10
+    ref_gate, ref = run_stream(norms, tau=2.5, gate_eps=0.0, window=10)
+    assert ref_gate.s_star == 38
+    for shift, scale in ((100.0, 1.0), (0.0, 1e-3), (5.0, 40.0)):
+        gate, recs = run_stream(shift + scale * norms, tau=2.5, gate_eps=0.0, window=10)
+        assert gate.s_star == ref_gate.s_star and len(recs) == len(ref)
+        for (t0, z0, mu0, s0), (t1, z1, mu1, s1) in zip(ref, recs):
+            assert t0 == t1
+            if not math.isnan(z0):
+                assert z1 == pytest.approx(z0, rel=1e-7, abs=1e-9)
+                assert mu1 == pytest.approx(shift + scale * mu0, rel=1e-12)
+                assert s1 == pytest.approx(scale * s0, rel=1e-7, abs=1e-12)

@@ -329,3 +329,60 @@ def test_bf16_rounding_matches_the_library_conversion():
     assert got[-6] == 0x3F80 and got[-5] == 0x3F82 and got[-3] == 0x7F80
     nan = ora.round_to_bf16(np.array([np.nan]))
     assert (nan[0] & 0x7F80) == 0x7F80 and (nan[0] & 0x007F) != 0
+
+
+# ---------------------------------------------------------------------------
+# invariances the mathematics fixes (no value is taken from any implementation)
+# ---------------------------------------------------------------------------
+def test_geometric_sum_recurrence_links_consecutive_depths():
+    """S_{K+1}(r) = 1 + r S_K(r) (Eq. (geom_sum_def)), and scale_K (1 + r) = S_K(r): the oracle's
+    scale factors for consecutive K must satisfy scale_{K+1} (1+r) = 1 + r scale_K (1+r).  A wrong
+    loop bound, a dropped term or a swapped numerator/denominator breaks it for some K."""
+    rng = np.random.default_rng(5)
+    r = np.concatenate([rng.uniform(-0.95, 2.5, 200), [-3.0, 0.0, 1.0, 7.5]])
+    for K in range(2, 12):
+        sk, sk1 = _scale(r, K), _scale(r, K + 1)
+        np.testing.assert_allclose(sk1 * (1.0 + r), 1.0 + r * sk * (1.0 + r), rtol=1e-11, atol=1e-12)
+
+
+def test_extrapolation_depends_on_the_gradients_only_through_their_ratio_and_is_linear_in_the_displacement():
+    rng = np.random.default_rng(6)
+    n = 300
+    th0 = rng.standard_normal(n)
+    d = 1e-2 * rng.standard_normal(n)
+    g0 = rng.standard_normal(n)
+    g1 = g0 * rng.uniform(-0.8, 1.6, n)
+    for K in (3, 5, 10):
+        base = ora.extrapolate(th0, th0 + d, g0, g1, K, 0.5, 1e-8)
+        for c in (1e-3, 7.0):                    # (g0, g1) -> (c g0, c g1): same ratio, same active set
+            same = ora.extrapolate(th0, th0 + d, c * g0, c * g1, K, 0.5, 1e-8 * min(c, 1.0))
+            np.testing.assert_allclose(same, base, rtol=1e-12, atol=1e-15)
+        dbl = ora.extrapolate(th0, th0 + 2.0 * d, g0, g1, K, 0.5, 1e-8)      # Eq. (blend_step): linear in theta2 - theta0
+        np.testing.assert_allclose(dbl - th0, 2.0 * (base - th0), rtol=1e-11, atol=1e-15)
+        neg = ora.extrapolate(th0, th0 + d, -g0, -g1, K, 0.5, 1e-8)          # a common sign drops out of g1 / g0
+        np.testing.assert_allclose(neg, base, rtol=1e-13, atol=0)
+
+
+def test_adam_update_is_invariant_to_the_scale_of_the_gradients_when_eps_is_zero():
+    """m / sqrt(v) is homogeneous of degree zero in the gradient history: with eps = 0 and no weight
+    decay, multiplying every gradient by c > 0 leaves every parameter where it was (the textbook
+    scale invariance of Adam).  It pins the pairing of m with sqrt(v), both bias corrections and
+    the place of eps."""
+    rng = np.random.default_rng(7)
+    n, steps = 64, 6
+    grads = [rng.standard_normal(n) for _ in range(steps)]
+    outs = []
+    for c in (1.0, 1e-4, 3e3):
+        opt = ora.OptCfg(kind="adamw", lr=1e-2, eps=0.0, weight_decay=0.0)
+        st = ora.State(np.linspace(-1.0, 1.0, n), opt)
+        for g in grads:
+            st.optim_step(c * g, False)
+        outs.append(st.theta.copy())
+    np.testing.assert_allclose(outs[1], outs[0], rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(outs[2], outs[0], rtol=1e-11, atol=1e-13)
+    # and with eps > 0 the invariance must break in the expected direction: tiny gradients move less
+    opt = ora.OptCfg(kind="adamw", lr=1e-2, eps=1e-3, weight_decay=0.0)
+    small, big = ora.State(np.zeros(n), opt), ora.State(np.zeros(n), opt)
+    small.optim_step(1e-4 * grads[0], False)
+    big.optim_step(grads[0], False)
+    assert np.all(np.abs(small.theta) < np.abs(big.theta))
